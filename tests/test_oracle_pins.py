@@ -1,0 +1,386 @@
+"""Pins for the CPU oracle: each test fixes a part of it to something other than itself.
+
+Sources of truth used here: the hand-worked examples under tests/golden/ (Eq. 1-7, 11, 12),
+closed forms, invariants the equations imply, brute force on tiny shapes written as explicit
+Python loops over unpacked operands, and numpy's float64 matmul on a special case.
+"""
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import oracle as O
+
+GOLD = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "worked_examples.json")))
+
+
+def unpack_pm1(bits, K):
+    """bits u8 [N,K/8] -> +-1 int array [N,K]; bit k%8 of byte k/8, 1 = +1."""
+    b = np.unpackbits(bits, axis=1, bitorder="little")[:, :K].astype(np.int64)
+    return 2 * b - 1
+
+
+# ---------------------------------------------------------------- worked examples (golden)
+
+def test_golden_binarize():
+    fx = GOLD["binarize_2x8"]
+    r = O.binarize(np.array(fx["W"], np.float32))
+    assert r["alpha"][0] == fx["alpha"]
+    assert r["beta"][0] == fx["beta"]
+    assert r["bits"].reshape(-1).tolist() == fx["bytes"]
+    assert r["rowsum"].reshape(-1).tolist() == fx["rowsum"]
+
+
+def test_golden_absmax_ties():
+    fx = GOLD["absmax_ties_noLN"]
+    r = O.quant_act(np.array([fx["x"]], np.float32), ln_eps=-1.0)
+    assert r["gamma"].reshape(-1)[0] == fx["gamma"]
+    assert r["codes"][0].tolist() == fx["codes"]
+
+
+def test_golden_eta():
+    fx = GOLD["eta_noLN"]
+    r = O.quant_act(np.array([fx["x"]], np.float32), mode=O.ETA, ln_eps=-1.0)
+    assert r["eta"].reshape(-1)[0] == fx["eta"]
+    assert r["gamma"].reshape(-1)[0] == fx["gamma"]
+    assert r["codes"][0].tolist() == fx["codes"]
+
+
+def test_golden_ln_absmax():
+    fx = GOLD["ln_absmax_1to8"]
+    r = O.quant_act(np.array([fx["x"]], np.float32), ln_eps=fx["ln_eps"])
+    assert abs(r["gamma"].reshape(-1)[0] - fx["gamma"]) < 1e-14
+    assert r["codes"][0].tolist() == fx["codes"]
+
+
+def test_golden_forward():
+    fb, fl, ff = GOLD["binarize_2x8"], GOLD["ln_absmax_1to8"], GOLD["forward_2x8"]
+    w = O.binarize(np.array(fb["W"], np.float32))
+    r = O.forward(np.array([fl["x"]], np.float32), w["bits"], w["beta"], ln_eps=0.0)
+    assert r["acc"].reshape(-1).tolist() == ff["acc"]
+    np.testing.assert_allclose(r["y"].reshape(-1), ff["y"], rtol=1e-14)
+
+
+# ---------------------------------------------------------------- binarization (Eq. 1-3, 12, 13)
+
+def test_sign_tie_is_minus_one():
+    # symmetric integer-valued W: alpha = 0 exactly; zeros must binarize to -1 (bit 0).
+    W = np.array([[-2, -1, 0, 0, 1, 2, 0, 0], [3, 0, -3, 0, 0, 0, 1, -1]], np.float32)
+    r = O.binarize(W)
+    assert r["alpha"][0] == 0.0
+    expect = np.where(W > 0, 1, -1)
+    assert (unpack_pm1(r["bits"], 8) == expect).all()
+
+
+def test_alpha_beta_closed_forms():
+    # arithmetic progression 1..N*K: alpha = (NK+1)/2, beta the same (all positive).
+    N, K = 4, 16
+    W = np.arange(1, N * K + 1, dtype=np.float32).reshape(N, K)
+    r = O.binarize(W)
+    assert r["alpha"][0] == (N * K + 1) / 2
+    assert r["beta"][0] == (N * K + 1) / 2
+    # +-c checkerboard: alpha = 0, beta = c, signs follow the pattern.
+    c = 0.375
+    P = np.where((np.add.outer(np.arange(N), np.arange(K)) % 2) == 0, c, -c).astype(np.float32)
+    r = O.binarize(P)
+    assert r["alpha"][0] == 0.0 and r["beta"][0] == c
+    assert (unpack_pm1(r["bits"], K) == np.sign(P)).all()
+    assert (r["rowsum"] == 0).all()
+
+
+def test_gaussian_closed_form_and_zero_centre():
+    rng = np.random.default_rng(5)
+    N, K, sigma = 512, 1024, 0.02
+    W = (rng.standard_normal((N, K)) * sigma).astype(np.float32)
+    r = O.binarize(W)
+    nk = N * K
+    assert abs(r["beta"][0] - sigma * math.sqrt(2 / math.pi)) < 4 / math.sqrt(nk) * sigma
+    assert abs(r["alpha"][0]) < 5 * sigma / math.sqrt(nk)
+    pm = unpack_pm1(r["bits"], K)
+    assert abs(pm.sum()) <= 6 * math.sqrt(nk)                       # zero-centred
+    assert (pm.sum(axis=1) == r["rowsum"][:, 0]).all()
+    # beta * ||W~||_1 = ||W||_1
+    l1 = np.abs(W.astype(np.float64)).sum()
+    assert abs(r["beta"][0] * np.abs(pm).sum() - l1) <= 1e-12 * l1
+    # mean against numpy's pairwise float64 mean
+    assert abs(r["alpha"][0] - W.astype(np.float64).mean()) < 1e-15
+
+
+def test_alpha_is_subtracted_not_added():
+    # all weights positive, so Sign(W) would be all +1; Sign(W - alpha) splits around the mean.
+    W = np.array([[1, 2, 3, 4, 5, 6, 7, 8]], np.float32)
+    r = O.binarize(W)
+    assert unpack_pm1(r["bits"], 8).reshape(-1).tolist() == [-1, -1, -1, -1, 1, 1, 1, 1]
+
+
+def test_group_binarize_matches_slices():
+    rng = np.random.default_rng(6)
+    N, K, G = 8, 64, 4
+    W = (rng.standard_normal((N, K)) * 0.02 + np.repeat(np.arange(G) * 0.01, K // G)).astype(np.float32)
+    r = O.binarize(W, G=G)
+    Kg = K // G
+    for g in range(G):
+        s = O.binarize(W[:, g * Kg:(g + 1) * Kg])
+        assert s["alpha"][0] == r["alpha"][g] and s["beta"][0] == r["beta"][g]
+        assert (s["bits"] == r["bits"][:, g * Kg // 8:(g + 1) * Kg // 8]).all()
+        assert (s["rowsum"][:, 0] == r["rowsum"][:, g]).all()
+    # group means really differ, so a whole-tensor alpha would give other bits
+    assert not (O.binarize(W)["bits"] == r["bits"]).all()
+
+
+def test_alpha_override():
+    W = np.array([[1, 2, 3, 4, 5, 6, 7, 8]], np.float32)
+    r = O.binarize(W, alpha_in=[6.5])
+    assert unpack_pm1(r["bits"], 8).reshape(-1).tolist() == [-1] * 6 + [1, 1]
+    assert r["beta"][0] == 4.5
+
+
+# ---------------------------------------------------------------- LN (Eq. 12, 15)
+
+def test_ln_moments_and_constant_row():
+    rng = np.random.default_rng(7)
+    M, K, eps = 5, 256, 1e-5
+    x = (rng.standard_normal((M, K)) * 3 + 1.5).astype(np.float32)
+    x[4] = 2.75                                                   # constant row
+    r = O.quant_act(x, ln_eps=eps, want_xhat=True)
+    xh = r["xhat"]
+    assert np.abs(xh.mean(axis=1)).max() < 1e-12
+    var = x.astype(np.float64).var(axis=1)
+    np.testing.assert_allclose(xh.var(axis=1)[:4], (var / (var + eps))[:4], rtol=1e-12)
+    assert (xh[4] == 0).all() and (r["codes"][4] == 0).all() and r["gamma"][4, 0] == 0.0
+    assert np.isfinite(xh).all()
+
+
+def test_ln_group_norm():
+    rng = np.random.default_rng(8)
+    M, K, G = 3, 128, 4
+    x = rng.standard_normal((M, K)).astype(np.float32) * np.repeat([1, 5, 0.2, 9], K // G).astype(np.float32)
+    r = O.quant_act(x, G=G, ln_eps=1e-5, want_xhat=True)
+    Kg = K // G
+    for g in range(G):
+        s = O.quant_act(np.ascontiguousarray(x[:, g * Kg:(g + 1) * Kg]), ln_eps=1e-5, want_xhat=True)
+        assert (s["xhat"] == r["xhat"][:, g * Kg:(g + 1) * Kg]).all()
+        assert (s["codes"] == r["codes"][:, g * Kg:(g + 1) * Kg]).all()
+        assert (s["gamma"][:, 0] == r["gamma"][:, g]).all()
+
+
+# ---------------------------------------------------------------- Quant (Eq. 4-6, 14)
+
+@pytest.mark.parametrize("gran", [O.PER_TOKEN, O.PER_TENSOR])
+def test_code_bounds_saturation_and_rounding_bound(gran):
+    rng = np.random.default_rng(9)
+    M, K = 16, 512
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    x[rng.random((M, K)) < 0.002] *= 20
+    r = O.quant_act(x, gran=gran, ln_eps=1e-5, want_xhat=True)
+    codes, xh = r["codes"].astype(np.int64), r["xhat"]
+    assert np.abs(codes).max() == 127                              # |code| <= Q_b - 1, reached
+    gam = r["gamma"][:, 0][:, None] if gran == O.PER_TOKEN else r["gamma"][0]
+    if gran == O.PER_TOKEN:
+        i = np.abs(xh).argmax(axis=1)
+        assert (np.abs(codes[np.arange(M), i]) == 127).all()       # the arg-max saturates
+        np.testing.assert_allclose(r["gamma"][:, 0], np.abs(xh).max(axis=1), rtol=0, atol=0)
+    else:
+        assert r["gamma"][0] == np.abs(xh).max()
+    gam = np.broadcast_to(gam, xh.shape)
+    err = np.abs(codes * gam / 128 - xh)
+    unsat = np.abs(xh * 128 / gam) <= 127.5
+    assert (err[unsat] <= gam[unsat] / 256 * (1 + 1e-12)).all()
+    assert (err <= gam / 128 * (1 + 1e-12)).all()
+    # sign of codes follows sign of xhat
+    assert (np.sign(codes) * np.sign(xh) >= 0).all()
+
+
+def test_eta_mode_range_and_endpoints():
+    rng = np.random.default_rng(10)
+    M, K = 8, 256
+    x = np.maximum(rng.standard_normal((M, K)), 0).astype(np.float32)
+    r = O.quant_act(x, mode=O.ETA, ln_eps=1e-5, want_xhat=True)
+    codes, xh = r["codes"], r["xhat"]
+    assert codes.min() == 0 and codes.max() == 127
+    rows = np.arange(M)
+    assert (codes[rows, xh.argmin(axis=1)] == 0).all()
+    assert (codes[rows, xh.argmax(axis=1)] == 127).all()
+    np.testing.assert_array_equal(r["eta"][:, 0], xh.min(axis=1))
+    np.testing.assert_array_equal(r["gamma"][:, 0], xh.max(axis=1) - xh.min(axis=1))
+    recon = codes * (r["gamma"][:, :1] / 128) + r["eta"][:, :1]
+    assert (np.abs(recon - xh) <= r["gamma"][:, :1] / 128 * (1 + 1e-12)).all()
+
+
+def test_half_to_even_ties_exact():
+    # gamma = 128 planted, LN skipped -> scale exactly 1.
+    vals = [0.5, 1.5, 2.5, 3.5, -0.5, -1.5, -2.5, -3.5, 126.5, -126.5, 127.5, 128.0, 0.0, 1.0, -1.0, 2.0]
+    x = np.array([vals], np.float32)
+    r = O.quant_act(x, ln_eps=-1.0)
+    assert r["codes"][0].tolist() == [0, 2, 2, 4, 0, -2, -2, -4, 126, -126, 127, 127, 0, 1, -1, 2]
+
+
+def test_per_tensor_gamma_is_global():
+    x = np.zeros((2, 8), np.float32)
+    x[0, 0], x[1, 3] = 4.0, -64.0
+    r = O.quant_act(x, gran=O.PER_TENSOR, ln_eps=-1.0)
+    assert r["gamma"].tolist() == [64.0]
+    assert r["codes"][0, 0] == 8 and r["codes"][1, 3] == -127
+    rt = O.quant_act(x, gran=O.PER_TOKEN, ln_eps=-1.0)
+    assert rt["gamma"][:, 0].tolist() == [4.0, 64.0] and rt["codes"][0, 0] == 127
+
+
+def test_zero_input_gives_zero_codes():
+    r = O.quant_act(np.zeros((2, 16), np.float32), ln_eps=1e-5)
+    assert (r["codes"] == 0).all() and (r["gamma"] == 0).all()
+    r = O.quant_act(np.zeros((2, 16), np.float32), mode=O.ETA, ln_eps=-1.0)
+    assert (r["codes"] == 0).all()
+
+
+# ---------------------------------------------------------------- matmul (Eq. 7)
+
+@pytest.mark.parametrize("M,N,K,G", [(1, 1, 8, 1), (3, 5, 16, 1), (4, 8, 64, 1), (2, 3, 64, 4)])
+def test_matmul_brute_force(M, N, K, G):
+    rng = np.random.default_rng(100 + K + G)
+    codes = rng.integers(-127, 128, (M, K)).astype(np.int8)
+    bits = rng.integers(0, 256, (N, K // 8)).astype(np.uint8)
+    acc = O.matmul(codes, bits, G=G)
+    Kg = K // G
+    for g in range(G):
+        for m in range(M):
+            for n in range(N):
+                s = 0
+                for k in range(g * Kg, (g + 1) * Kg):
+                    bit = (int(bits[n, k // 8]) >> (k % 8)) & 1
+                    s += (1 if bit else -1) * int(codes[m, k])
+                assert acc[g, m, n] == s
+
+
+def test_matmul_all_plus_all_minus_and_one_hot():
+    rng = np.random.default_rng(11)
+    M, N, K = 4, 6, 64
+    codes = rng.integers(-127, 128, (M, K)).astype(np.int8)
+    plus = np.full((N, K // 8), 0xFF, np.uint8)
+    assert (O.matmul(codes, plus)[0] == codes.astype(np.int64).sum(axis=1)[:, None]).all()
+    assert (O.matmul(codes, np.zeros_like(plus))[0] == -codes.astype(np.int64).sum(axis=1)[:, None]).all()
+    # one-hot code rows read back W~[n,k]*127 for every k: pins bit order and K-major packing.
+    bits = rng.integers(0, 256, (N, K // 8)).astype(np.uint8)
+    onehot = (np.eye(K) * 127).astype(np.int8)
+    acc = O.matmul(onehot, bits)[0]                                 # [K, N]
+    assert (acc.T == 127 * unpack_pm1(bits, K)).all()
+
+
+def test_matmul_against_float64_gemm_and_samples():
+    rng = np.random.default_rng(12)
+    M, N, K, G = 33, 70, 256, 2
+    codes = rng.integers(-127, 128, (M, K)).astype(np.int8)
+    bits = rng.integers(0, 256, (N, K // 8)).astype(np.uint8)
+    acc = O.matmul(codes, bits, G=G)
+    pm = unpack_pm1(bits, K).astype(np.float64)
+    Kg = K // G
+    for g in range(G):
+        ref = codes[:, g * Kg:(g + 1) * Kg].astype(np.float64) @ pm[:, g * Kg:(g + 1) * Kg].T
+        assert (acc[g] == ref).all()
+    ms = rng.integers(0, M, 50)
+    ns = rng.integers(0, N, 50)
+    s = O.matmul_samples(codes, bits, ms, ns, G=G)
+    for g in range(G):
+        assert (s[:, g] == acc[g, ms, ns]).all()
+
+
+def test_matmul_is_not_transposed():
+    # M != N and an asymmetric pattern: swapping operands or indices cannot pass.
+    codes = np.zeros((2, 8), np.int8)
+    codes[0, 0], codes[1, 7] = 5, 9
+    bits = np.zeros((3, 1), np.uint8)
+    bits[1, 0] = 0x01      # row 1: +1 at k = 0
+    bits[2, 0] = 0x80      # row 2: +1 at k = 7
+    acc = O.matmul(codes, bits)[0]
+    assert acc.shape == (2, 3)
+    assert acc.tolist() == [[-5, 5, -5], [-9, -9, 9]]
+
+
+# ---------------------------------------------------------------- dequant / forward (Eq. 11)
+
+def test_forward_equals_staged_and_linearity_bound():
+    rng = np.random.default_rng(13)
+    M, N, K = 16, 48, 1024
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float32)
+    w = O.binarize(W)
+    f = O.forward(x, w["bits"], w["beta"], ln_eps=1e-5)
+    q = O.quant_act(x, ln_eps=1e-5, want_xhat=True)
+    acc = O.matmul(q["codes"], w["bits"])
+    y = O.dequant(acc, w["beta"], q["gamma"])
+    assert (f["y"] == y).all() and (f["codes"] == q["codes"]).all()
+    # Eq. 11 written out with numpy on the oracle's own integer results
+    y_np = acc[0].astype(np.float64) * w["beta"][0] * q["gamma"] / 128.0
+    np.testing.assert_allclose(y, y_np, rtol=1e-14)
+    # y approximates beta * W~ xhat with uniform-quantisation-noise error
+    pm = unpack_pm1(w["bits"], K).astype(np.float64)
+    exact = w["beta"][0] * q["xhat"] @ pm.T
+    rms_err = np.sqrt(((y - exact) ** 2).mean())
+    bound = (q["gamma"].max() / (128 * math.sqrt(12))) * w["beta"][0] * math.sqrt(K) * 1.2
+    assert rms_err <= bound
+    assert rms_err >= 0.5 * (q["gamma"].min() / (128 * math.sqrt(12))) * w["beta"][0] * math.sqrt(K)
+
+
+def test_variance_argument():
+    # Eq. 8-10: Var(y) ~ K * beta^2 * E[xhat_q^2]; with LN that is ~ K beta^2.
+    rng = np.random.default_rng(14)
+    M, N, K = 32, 256, 4096
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float32)
+    w = O.binarize(W)
+    f = O.forward(x, w["bits"], w["beta"], ln_eps=1e-5)
+    rms = np.sqrt((f["y"] ** 2).mean())
+    assert abs(rms / (w["beta"][0] * math.sqrt(K)) - 1.0) < 0.05
+
+
+def test_group_forward_is_sum_of_slices():
+    rng = np.random.default_rng(15)
+    M, N, K, G = 6, 10, 256, 4
+    x = np.maximum(rng.standard_normal((M, K)), 0).astype(np.float32)
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float32)
+    Kg = K // G
+    for mode in (O.ABSMAX, O.ETA):
+        for gran in (O.PER_TOKEN, O.PER_TENSOR):
+            w = O.binarize(W, G=G)
+            f = O.forward(x, w["bits"], w["beta"], G=G, mode=mode, gran=gran, ln_eps=1e-5)
+            total = np.zeros((M, N))
+            for g in range(G):
+                ws = O.binarize(W[:, g * Kg:(g + 1) * Kg])
+                fs = O.forward(np.ascontiguousarray(x[:, g * Kg:(g + 1) * Kg]), ws["bits"], ws["beta"],
+                               mode=mode, gran=gran, ln_eps=1e-5)
+                assert (fs["acc"][0] == f["acc"][g]).all()
+                total += fs["y"]
+            np.testing.assert_allclose(f["y"], total, rtol=1e-13, atol=1e-15)
+    # G = 1 is the ungrouped layer
+    w1 = O.binarize(W, G=1)
+    assert (O.forward(x, w1["bits"], w1["beta"], G=1)["y"] == O.forward(x, w1["bits"], w1["beta"])["y"]).all()
+
+
+def test_eta_correction_restores_unshifted_product():
+    rng = np.random.default_rng(16)
+    M, N, K = 4, 12, 512
+    x = np.maximum(rng.standard_normal((M, K)), 0).astype(np.float32)
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float32)
+    w = O.binarize(W)
+    lit = O.forward(x, w["bits"], w["beta"], mode=O.ETA, ln_eps=1e-5)
+    cor = O.forward(x, w["bits"], w["beta"], mode=O.ETA, ln_eps=1e-5, rowsum=w["rowsum"], eta_correction=True)
+    diff = cor["y"] - lit["y"]
+    expect = lit["eta"][:, :1] * w["beta"][0] * w["rowsum"][:, 0][None, :]
+    np.testing.assert_allclose(diff, expect, rtol=1e-12, atol=1e-15)
+    q = O.quant_act(x, mode=O.ETA, ln_eps=1e-5, want_xhat=True)
+    exact = w["beta"][0] * q["xhat"] @ unpack_pm1(w["bits"], K).astype(np.float64).T
+    assert np.sqrt(((cor["y"] - exact) ** 2).mean()) < 0.02 * np.sqrt((exact ** 2).mean())
+
+
+def test_dequant_scale_is_qb_128_not_127():
+    acc = np.array([[[128]]], np.int32)
+    y = O.dequant(acc, [0.5], [[2.0]])
+    assert y[0, 0] == 128 * 0.5 * 2.0 / 128
+
+
+def test_bad_shapes_are_rejected():
+    with pytest.raises(ValueError):
+        O.binarize(np.zeros((2, 12), np.float32))            # K % 8 != 0
+    with pytest.raises(ValueError):
+        O.quant_act(np.zeros((2, 16), np.float32), G=4)      # K % (8 G) != 0
