@@ -1,0 +1,154 @@
+/*
+ * bitlinear.h - C ABI of the B200 (sm_100a) BitLinear forward library.
+ *
+ * BitLinear (BitNet, Sec. 2.1, Eq. 11):   y = W~ . Quant(LN(x)) . beta.gamma / Q_b
+ *   step 1  LN(x) = (x - E x) / sqrt(Var x + eps)                         Eq. 12 (per group: Eq. 15)
+ *   step 2  x~ = Clip(round(x^.Q_b/gamma), -(Q_b-1), Q_b-1), gamma = max|x^|   Eq. 4-5
+ *           or Clip(round((x^-eta).Q_b/gamma), 0, Q_b-1), eta = min x^         Eq. 6
+ *   step 3  W~ = Sign(W - alpha), alpha = mean W, beta = mean|W|          Eq. 1-3, 12 (per group: Eq. 13)
+ *   step 4  acc = W~ x~ in exact integers, rescaled by beta.gamma/Q_b     Eq. 7, 11
+ * Symbols follow the paper: M tokens, K input features (the contraction and the group
+ * dimension), N output features, G groups along K (K_g = K/G), b = 8 bits, Q_b = 2^(b-1) = 128.
+ *
+ * Conventions that hold for every entry point unless it says otherwise
+ *   - Every data pointer is a DEVICE pointer owned by the caller; matrices are dense row-major;
+ *     base addresses are 16-byte aligned (BL_ERR_ALIGN otherwise).
+ *   - The library allocates nothing and keeps no state between calls.  Scratch comes from the
+ *     caller as (ws, ws_bytes); ask bitlinear_workspace_bytes() for the size.  The workspace
+ *     may be reused by the next call on the same stream; it holds nothing the caller needs
+ *     except the status word read by bitlinear_ws_status().
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default
+ *     stream) and never synchronise.
+ *   - Errors are detected on the host before any launch and returned as a bl_status; nothing
+ *     is launched when the status is not BL_OK.  Kernels never trap or print.  A device-side
+ *     wait that runs out of its iteration limit records BL_ERR_TIMEOUT in the workspace
+ *     status word; outputs of that call are then undefined.
+ *   - Rounding to integer codes and to 16-bit outputs is round-half-to-even.
+ *   - Requirements on shapes: K % (8*G) == 0, 1 <= G <= BL_MAX_GROUPS, b == 8
+ *     (Sec. 2.1 leaves other widths to future work: BL_ERR_UNSUPPORTED).
+ */
+#ifndef BITLINEAR_H_
+#define BITLINEAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define BL_MAX_GROUPS 64
+
+typedef enum {
+  BL_OK = 0,
+  BL_ERR_NULL = 1,        /* a required pointer is NULL */
+  BL_ERR_SHAPE = 2,       /* a size is non-positive or breaks a divisibility rule */
+  BL_ERR_ALIGN = 3,       /* a pointer is not 16-byte aligned */
+  BL_ERR_UNSUPPORTED = 4, /* b != 8, unknown enum value, or layout not accepted by this call */
+  BL_ERR_WORKSPACE = 5,   /* ws is NULL or smaller than bitlinear_workspace_bytes() */
+  BL_ERR_CUDA = 6,        /* a CUDA runtime call (launch, attribute, tensor map) failed */
+  BL_ERR_TIMEOUT = 7      /* a bounded device-side wait expired (read via bitlinear_ws_status) */
+} bl_status;
+
+typedef enum { BL_F32 = 0, BL_F16 = 1, BL_BF16 = 2 } bl_dtype;
+
+/* Eq. 4-5 (signed codes in [-127,127]) or Eq. 6 (eta-shifted codes in [0,127]). */
+typedef enum { BL_ABSMAX = 0, BL_ETA = 1 } bl_quant_mode;
+
+/* Scope of gamma/eta (Sec. 2.1: per tensor in training, per token in inference).
+ * PER_TENSOR: gamma, eta have G entries.  PER_TOKEN: M*G entries, index m*G + g. */
+typedef enum { BL_PER_TENSOR = 0, BL_PER_TOKEN = 1 } bl_gran;
+
+/* Storage order of the 1-bit weights W~ (bit = 1 means +1).
+ *   CANONICAL  u8 [N, K/8]; weight k of row n is bit (k % 8) of byte n*K/8 + k/8.  Accepted by
+ *              every entry point except gemv_decode; shapes are unrestricted.
+ *   PREFILL    the same bits re-tiled for the tensor-core GEMM: blocks of 128 rows x 128
+ *              weights, rows and K padded up to multiples of 128 (see bitlinear_packed_bytes and
+ *              bitlinear_layout_index).  Needs K % 16 == 0 and K_g % 128 == 0.
+ *   DECODE     the same bits re-ordered for the batch-1 GEMV.  Needs K % 256 == 0, N % 16 == 0. */
+typedef enum { BL_LAYOUT_CANONICAL = 0, BL_LAYOUT_PREFILL = 1, BL_LAYOUT_DECODE = 2 } bl_layout;
+
+typedef enum {
+  BL_OP_BINARIZE_PACK = 0,
+  BL_OP_QUANT_ACT = 1,
+  BL_OP_FORWARD = 2,
+  BL_OP_MATMUL_I32 = 3
+} bl_op;
+
+/* Human-readable name of a status code (static string, never NULL). */
+const char* bitlinear_status_string(bl_status st);
+
+/* Bytes of scratch the given entry point needs for these sizes (0 on invalid sizes). */
+size_t bitlinear_workspace_bytes(bl_op op, int64_t M, int64_t N, int64_t K, int G);
+
+/* Bytes of the packed weight buffer for a layout (includes PREFILL padding); 0 if invalid. */
+size_t bitlinear_packed_bytes(bl_layout layout, int64_t N, int64_t K);
+
+/* Where weight (n, k) lives in a packed buffer of the given layout: writes the byte offset
+ * and the bit number.  Host-only helper that documents the private layouts; tests use it to
+ * map PREFILL/DECODE buffers back to CANONICAL.  Returns BL_ERR_SHAPE when out of range. */
+bl_status bitlinear_layout_index(bl_layout layout, int64_t N, int64_t K, int64_t n, int64_t k,
+                                 int64_t* byte_offset, int* bit);
+
+/* Step 3, Eq. 1-3, 12, 13: alpha_g, beta_g over the K-slice g of all N rows, then
+ * W~ = Sign(W - alpha_g) with Sign(0) = -1, packed 1 bit per weight.
+ *   W         [N,K] of dtype wt (read twice).
+ *   alpha_in  NULL, or G device floats used in place of the computed means (lets a caller
+ *             fix alpha, e.g. to isolate the sign-and-pack step).
+ *   W_packed  bitlinear_packed_bytes(layout,N,K) bytes, fully overwritten.
+ *   alpha, beta  [G] fp32 outputs (the means in fp64, rounded once).
+ *   rowsum    NULL or int32 [N,G]: sum over the group of W~[n,k] (used by eta_correction).
+ * Sums are accumulated in fp64 in a fixed order, so results are run-to-run identical; the sign
+ * test compares W against the fp64 mean exactly.  Workspace: BL_OP_BINARIZE_PACK. */
+bl_status bitlinear_binarize_pack(const void* W, bl_dtype wt, int64_t N, int64_t K, int G,
+                                  bl_layout layout, const float* alpha_in, uint8_t* W_packed,
+                                  float* alpha, float* beta, int32_t* rowsum, void* ws,
+                                  size_t ws_bytes, void* stream);
+
+/* Steps 1-2, Eq. 12/15 then Eq. 4-6/14, b = 8.
+ *   x      [M,K] of dtype xt.
+ *   ln_eps LN epsilon; a negative value skips LN (codes are taken from x itself).
+ *   x_q    int8 [M,K] codes.   gamma, eta: fp32, sized by gran (eta may be NULL for BL_ABSMAX).
+ * gamma == 0 (constant input) yields all-zero codes, never NaN.  PER_TOKEN is one pass over x;
+ * PER_TENSOR is two (statistics, then codes).  Workspace: BL_OP_QUANT_ACT. */
+bl_status bitlinear_quant_act(const void* x, bl_dtype xt, int64_t M, int64_t K, int G, int b,
+                              bl_quant_mode mode, bl_gran gran, float ln_eps, int8_t* x_q,
+                              float* gamma, float* eta, void* ws, size_t ws_bytes, void* stream);
+
+/* Steps 1, 2, 4, Eq. 11: y = (W~ x~) . beta_g gamma / Q_b summed over groups in ascending order.
+ *   eta_correction != 0 (BL_ETA only) adds eta.beta_g.rowsum[n,g], which undoes the shift of
+ *   Eq. 6 in the output; 0 is Eq. 11 as printed.
+ *   W_packed  CANONICAL (any shape, plain CUDA-core kernel) or PREFILL (tcgen05 tensor-core
+ *             kernel); beta [G] and rowsum [N,G] as produced by bitlinear_binarize_pack.
+ *   y      [M,N] of dtype yt.
+ * Workspace: BL_OP_FORWARD (holds the int8 codes, gamma, eta and the status word). */
+bl_status bitlinear_forward(const void* x, bl_dtype xt, int64_t M, int64_t K, int64_t N, int G,
+                            int b, bl_quant_mode mode, bl_gran gran, float ln_eps,
+                            int eta_correction, const uint8_t* W_packed, bl_layout layout,
+                            const float* beta, const int32_t* rowsum, void* y, bl_dtype yt,
+                            void* ws, size_t ws_bytes, void* stream);
+
+/* Step 4 alone, Eq. 7: acc[g,m,n] = sum over k in group g of W~[n,k] . x_q[m,k], exact int32.
+ * The parity hook for "accumulators are bit-exact when fed given codes".
+ *   x_q [M,K] int8;  acc int32 [G,M,N].  Layout CANONICAL or PREFILL as for bitlinear_forward.
+ * Workspace: BL_OP_MATMUL_I32. */
+bl_status bitlinear_matmul_i32(const int8_t* x_q, int64_t M, int64_t K, int64_t N, int G,
+                               const uint8_t* W_packed, bl_layout layout, int32_t* acc, void* ws,
+                               size_t ws_bytes, void* stream);
+
+/* Steps 1, 2, 4 for one token (M = 1), fused in a single kernel that streams the packed
+ * weights once; Eq. 11 with per-token gamma.  W_packed must be in DECODE layout.
+ *   x [K] of dtype xt;  y [N] of dtype yt.  No workspace, no device-side waits. */
+bl_status bitlinear_gemv_decode(const void* x, bl_dtype xt, int64_t K, int64_t N, int G, int b,
+                                bl_quant_mode mode, float ln_eps, int eta_correction,
+                                const uint8_t* W_packed, const float* beta,
+                                const int32_t* rowsum, void* y, bl_dtype yt, void* stream);
+
+/* Synchronises `stream`, then reads the status word a previous bitlinear_forward or
+ * bitlinear_matmul_i32 call left in `ws`.  BL_OK, BL_ERR_TIMEOUT, or BL_ERR_CUDA. */
+bl_status bitlinear_ws_status(const void* ws, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BITLINEAR_H_ */

@@ -1,0 +1,206 @@
+"""Thin Python binding of the BitLinear C ABI (include/bitlinear.h): argument marshalling only.
+
+Every function here has the name of the C entry point it calls.  torch supplies device memory
+and the current CUDA stream; every step of the computation runs in the library's kernels.
+There is no CPU path: a missing or unloadable library raises at first use.
+"""
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libbitlinear_b200.so")
+
+# enums of include/bitlinear.h
+OK = 0
+F32, F16, BF16 = 0, 1, 2
+ABSMAX, ETA = 0, 1
+PER_TENSOR, PER_TOKEN = 0, 1
+CANONICAL, PREFILL, DECODE = 0, 1, 2
+OP_BINARIZE_PACK, OP_QUANT_ACT, OP_FORWARD, OP_MATMUL_I32 = 0, 1, 2, 3
+MAX_GROUPS = 64
+
+EXPORTS = [
+    "bitlinear_status_string", "bitlinear_workspace_bytes", "bitlinear_packed_bytes",
+    "bitlinear_layout_index", "bitlinear_binarize_pack", "bitlinear_quant_act",
+    "bitlinear_forward", "bitlinear_matmul_i32", "bitlinear_gemv_decode", "bitlinear_ws_status",
+]
+
+_DTYPES = {torch.float32: F32, torch.float16: F16, torch.bfloat16: BF16}
+_lib = None
+
+
+class BitLinearError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = int(code)
+        super().__init__(f"{where}: {status_string(code)} (bl_status {int(code)})")
+
+
+def lib():
+    """Load the CUDA library (built in-tree by paper_2310_11453_b200.build); fail loudly."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2310_11453_b200.build` "
+                              "(there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        i64, vp, ci, sz = C.c_int64, C.c_void_p, C.c_int, C.c_size_t
+        L.bitlinear_status_string.restype = C.c_char_p
+        L.bitlinear_status_string.argtypes = [ci]
+        L.bitlinear_workspace_bytes.restype = sz
+        L.bitlinear_workspace_bytes.argtypes = [ci, i64, i64, i64, ci]
+        L.bitlinear_packed_bytes.restype = sz
+        L.bitlinear_packed_bytes.argtypes = [ci, i64, i64]
+        L.bitlinear_layout_index.restype = ci
+        L.bitlinear_layout_index.argtypes = [ci, i64, i64, i64, i64, C.POINTER(i64), C.POINTER(ci)]
+        L.bitlinear_binarize_pack.restype = ci
+        L.bitlinear_binarize_pack.argtypes = [vp, ci, i64, i64, ci, ci, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.bitlinear_quant_act.restype = ci
+        L.bitlinear_quant_act.argtypes = [vp, ci, i64, i64, ci, ci, ci, ci, C.c_float, vp, vp, vp, vp, sz, vp]
+        L.bitlinear_forward.restype = ci
+        L.bitlinear_forward.argtypes = [vp, ci, i64, i64, i64, ci, ci, ci, ci, C.c_float, ci, vp, ci,
+                                        vp, vp, vp, ci, vp, sz, vp]
+        L.bitlinear_matmul_i32.restype = ci
+        L.bitlinear_matmul_i32.argtypes = [vp, i64, i64, i64, ci, vp, ci, vp, vp, sz, vp]
+        L.bitlinear_gemv_decode.restype = ci
+        L.bitlinear_gemv_decode.argtypes = [vp, ci, i64, i64, ci, ci, ci, C.c_float, ci, vp, vp, vp,
+                                            vp, ci, vp]
+        L.bitlinear_ws_status.restype = ci
+        L.bitlinear_ws_status.argtypes = [vp, vp]
+        _lib = L
+    return _lib
+
+
+def status_string(code) -> str:
+    return lib().bitlinear_status_string(int(code)).decode()
+
+
+def _check(code, where):
+    if code != OK:
+        raise BitLinearError(code, where)
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dt(t):
+    try:
+        return _DTYPES[t.dtype]
+    except KeyError:
+        raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def workspace_bytes(op, M, N, K, G) -> int:
+    return int(lib().bitlinear_workspace_bytes(op, M, N, K, G))
+
+
+def packed_bytes(layout, N, K) -> int:
+    return int(lib().bitlinear_packed_bytes(layout, N, K))
+
+
+def layout_index(layout, N, K, n, k):
+    off, bit = C.c_int64(0), C.c_int(0)
+    _check(lib().bitlinear_layout_index(layout, N, K, n, k, C.byref(off), C.byref(bit)), "layout_index")
+    return off.value, bit.value
+
+
+def _ws(nbytes, device, ws=None):
+    if ws is not None:
+        return ws
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def binarize_pack(W, G=1, layout=CANONICAL, alpha_in=None, want_rowsum=True, out=None, ws=None):
+    """bitlinear_binarize_pack.  W [N,K] on the GPU.  Returns dict(W_packed u8, alpha, beta [G] f32,
+    rowsum [N,G] i32 or None).  `out` may carry preallocated tensors under the same keys."""
+    N, K = W.shape
+    dev = W.device
+    nbytes = packed_bytes(layout, N, K)
+    out = dict(out or {})
+    packed = out.get("W_packed")
+    if packed is None:
+        packed = torch.empty(max(nbytes, 16), dtype=torch.uint8, device=dev)
+    alpha = out.get("alpha", None)
+    alpha = alpha if alpha is not None else torch.empty(G, dtype=torch.float32, device=dev)
+    beta = out.get("beta", None)
+    beta = beta if beta is not None else torch.empty(G, dtype=torch.float32, device=dev)
+    rowsum = out.get("rowsum", None)
+    if rowsum is None and want_rowsum:
+        rowsum = torch.empty((N, G), dtype=torch.int32, device=dev)
+    ws = _ws(workspace_bytes(OP_BINARIZE_PACK, 1, N, K, G), dev, ws)
+    code = lib().bitlinear_binarize_pack(_ptr(W), _dt(W), N, K, G, layout, _ptr(alpha_in), _ptr(packed),
+                                         _ptr(alpha), _ptr(beta), _ptr(rowsum), _ptr(ws), ws.numel(),
+                                         _stream())
+    _check(code, "bitlinear_binarize_pack")
+    return dict(W_packed=packed, alpha=alpha, beta=beta, rowsum=rowsum, layout=layout, N=N, K=K, G=G)
+
+
+def quant_act(x, G=1, mode=ABSMAX, gran=PER_TOKEN, ln_eps=1e-5, b=8, out=None, ws=None):
+    """bitlinear_quant_act.  x [M,K].  Returns dict(x_q i8 [M,K], gamma, eta f32)."""
+    M, K = x.shape
+    dev = x.device
+    out = dict(out or {})
+    ns = (M, G) if gran == PER_TOKEN else (G,)
+    x_q = out.get("x_q")
+    x_q = x_q if x_q is not None else torch.empty((M, K), dtype=torch.int8, device=dev)
+    gamma = out.get("gamma")
+    gamma = gamma if gamma is not None else torch.empty(ns, dtype=torch.float32, device=dev)
+    eta = out.get("eta")
+    eta = eta if eta is not None else torch.zeros(ns, dtype=torch.float32, device=dev)
+    ws = _ws(workspace_bytes(OP_QUANT_ACT, M, 1, K, G), dev, ws)
+    code = lib().bitlinear_quant_act(_ptr(x), _dt(x), M, K, G, b, mode, gran, float(ln_eps), _ptr(x_q),
+                                     _ptr(gamma), _ptr(eta), _ptr(ws), ws.numel(), _stream())
+    _check(code, "bitlinear_quant_act")
+    return dict(x_q=x_q, gamma=gamma, eta=eta)
+
+
+def forward(x, W_packed, beta, N, G=1, mode=ABSMAX, gran=PER_TOKEN, ln_eps=1e-5, layout=CANONICAL,
+            rowsum=None, eta_correction=False, out_dtype=None, b=8, y=None, ws=None):
+    """bitlinear_forward.  x [M,K]; returns y [M,N] of out_dtype (default: x.dtype)."""
+    M, K = x.shape
+    dev = x.device
+    if y is None:
+        y = torch.empty((M, N), dtype=out_dtype or x.dtype, device=dev)
+    ws = _ws(workspace_bytes(OP_FORWARD, M, N, K, G), dev, ws)
+    code = lib().bitlinear_forward(_ptr(x), _dt(x), M, K, N, G, b, mode, gran, float(ln_eps),
+                                   1 if eta_correction else 0, _ptr(W_packed), layout, _ptr(beta),
+                                   _ptr(rowsum), _ptr(y), _dt(y), _ptr(ws), ws.numel(), _stream())
+    _check(code, "bitlinear_forward")
+    return y
+
+
+def matmul_i32(x_q, W_packed, N, G=1, layout=CANONICAL, acc=None, ws=None):
+    """bitlinear_matmul_i32.  x_q i8 [M,K]; returns acc i32 [G,M,N]."""
+    M, K = x_q.shape
+    dev = x_q.device
+    if acc is None:
+        acc = torch.empty((G, M, N), dtype=torch.int32, device=dev)
+    ws = _ws(workspace_bytes(OP_MATMUL_I32, M, N, K, G), dev, ws)
+    code = lib().bitlinear_matmul_i32(_ptr(x_q), M, K, N, G, _ptr(W_packed), layout, _ptr(acc), _ptr(ws),
+                                      ws.numel(), _stream())
+    _check(code, "bitlinear_matmul_i32")
+    return acc
+
+
+def gemv_decode(x, W_packed, beta, N, G=1, mode=ABSMAX, ln_eps=1e-5, rowsum=None,
+                eta_correction=False, out_dtype=None, b=8, y=None):
+    """bitlinear_gemv_decode.  x [K] or [1,K]; W_packed in DECODE layout; returns y [N]."""
+    K = x.numel()
+    if y is None:
+        y = torch.empty(N, dtype=out_dtype or x.dtype, device=x.device)
+    code = lib().bitlinear_gemv_decode(_ptr(x), _dt(x), K, N, G, b, mode, float(ln_eps),
+                                       1 if eta_correction else 0, _ptr(W_packed), _ptr(beta),
+                                       _ptr(rowsum), _ptr(y), _dt(y), _stream())
+    _check(code, "bitlinear_gemv_decode")
+    return y
+
+
+def ws_status(ws) -> int:
+    """bitlinear_ws_status: synchronises the current stream and returns the status word's verdict."""
+    return int(lib().bitlinear_ws_status(_ptr(ws), _stream()))

@@ -1,0 +1,225 @@
+// extern "C" entry points: argument validation on the host, workspace carving, launches.
+// Nothing here allocates device memory or synchronises (bitlinear_ws_status excepted).
+#include "common.cuh"
+
+namespace {
+
+using namespace bl;
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t round256(size_t v) { return (v + 255) & ~size_t(255); }
+inline bool valid_dtype(int t) { return t == BL_F32 || t == BL_F16 || t == BL_BF16; }
+
+// Common shape rules: sizes positive, 1 <= G <= BL_MAX_GROUPS, K % (8 G) == 0.
+inline bl_status check_kg(int64_t K, int G) {
+  if (K <= 0 || G < 1) return BL_ERR_SHAPE;
+  if (G > BL_MAX_GROUPS) return BL_ERR_UNSUPPORTED;
+  if (K % (8 * (int64_t)G) != 0) return BL_ERR_SHAPE;
+  return BL_OK;
+}
+
+constexpr size_t kStatusBytes = 256;   // status word lives at the start of a GEMM workspace
+
+struct ForwardWs {                     // carving of the BL_OP_FORWARD workspace
+  size_t status, codes, gamma, eta, quant, total;
+};
+ForwardWs carve_forward(int64_t M, int64_t K, int G) {
+  ForwardWs w;
+  size_t off = 0;
+  w.status = off; off += kStatusBytes;
+  w.codes = off;  off += round256((size_t)M * (size_t)K);
+  w.gamma = off;  off += round256((size_t)M * (size_t)G * sizeof(float));
+  w.eta = off;    off += round256((size_t)M * (size_t)G * sizeof(float));
+  w.quant = off;  off += round256(quant_ws_bytes(M, G));
+  w.total = off;
+  return w;
+}
+
+bl_status check_layout_for_gemm(bl_layout layout, int64_t M, int64_t K, int64_t N, int G) {
+  if (layout == BL_LAYOUT_CANONICAL) return BL_OK;
+  if (layout == BL_LAYOUT_PREFILL) return gemm_tc_supported(M, K, N, G) ? BL_OK : BL_ERR_SHAPE;
+  return BL_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* bitlinear_status_string(bl_status st) {
+  switch (st) {
+    case BL_OK: return "ok";
+    case BL_ERR_NULL: return "null pointer";
+    case BL_ERR_SHAPE: return "invalid shape";
+    case BL_ERR_ALIGN: return "pointer not 16-byte aligned";
+    case BL_ERR_UNSUPPORTED: return "unsupported option";
+    case BL_ERR_WORKSPACE: return "workspace missing or too small";
+    case BL_ERR_CUDA: return "CUDA runtime error";
+    case BL_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+size_t bitlinear_workspace_bytes(bl_op op, int64_t M, int64_t N, int64_t K, int G) {
+  (void)N;
+  if (check_kg(K, G) != BL_OK) return 0;
+  switch (op) {
+    case BL_OP_BINARIZE_PACK: return round256(pack_ws_bytes(G));
+    case BL_OP_QUANT_ACT: return M > 0 ? round256(quant_ws_bytes(M, G)) : 0;
+    case BL_OP_FORWARD: return M > 0 ? carve_forward(M, K, G).total : 0;
+    case BL_OP_MATMUL_I32: return kStatusBytes;
+  }
+  return 0;
+}
+
+size_t bitlinear_packed_bytes(bl_layout layout, int64_t N, int64_t K) {
+  if (N <= 0 || K <= 0 || K % 8 != 0) return 0;
+  switch (layout) {
+    case BL_LAYOUT_CANONICAL: return (size_t)(N * (K / 8));
+    case BL_LAYOUT_PREFILL: return K % 16 == 0 ? (size_t)prefill_bytes(N, K) : 0;
+    case BL_LAYOUT_DECODE: return (K % 256 == 0 && N % 16 == 0) ? (size_t)(N * (K / 8)) : 0;
+  }
+  return 0;
+}
+
+bl_status bitlinear_layout_index(bl_layout layout, int64_t N, int64_t K, int64_t n, int64_t k,
+                                 int64_t* byte_offset, int* bit) {
+  if (!byte_offset || !bit) return BL_ERR_NULL;
+  if (bitlinear_packed_bytes(layout, N, K) == 0 || n < 0 || n >= N || k < 0 || k >= K)
+    return BL_ERR_SHAPE;
+  switch (layout) {
+    case BL_LAYOUT_CANONICAL: *byte_offset = n * (K / 8) + k / 8; *bit = (int)(k % 8); break;
+    case BL_LAYOUT_PREFILL: prefill_index(K, n, k, byte_offset, bit); break;
+    case BL_LAYOUT_DECODE: decode_index(K, n, k, byte_offset, bit); break;
+  }
+  return BL_OK;
+}
+
+bl_status bitlinear_binarize_pack(const void* W, bl_dtype wt, int64_t N, int64_t K, int G,
+                                  bl_layout layout, const float* alpha_in, uint8_t* W_packed,
+                                  float* alpha, float* beta, int32_t* rowsum, void* ws,
+                                  size_t ws_bytes, void* stream) {
+  if (!W || !W_packed || !alpha || !beta) return BL_ERR_NULL;
+  if (N <= 0) return BL_ERR_SHAPE;
+  bl_status st = check_kg(K, G);
+  if (st != BL_OK) return st;
+  if (!valid_dtype(wt)) return BL_ERR_UNSUPPORTED;
+  if (layout != BL_LAYOUT_CANONICAL && layout != BL_LAYOUT_PREFILL && layout != BL_LAYOUT_DECODE)
+    return BL_ERR_UNSUPPORTED;
+  if (bitlinear_packed_bytes(layout, N, K) == 0) return BL_ERR_SHAPE;
+  if (layout == BL_LAYOUT_PREFILL && (K / G) % 128 != 0) return BL_ERR_SHAPE;
+  if (!aligned16(W) || !aligned16(W_packed)) return BL_ERR_ALIGN;
+  if (!ws || ws_bytes < bitlinear_workspace_bytes(BL_OP_BINARIZE_PACK, 1, N, K, G)) return BL_ERR_WORKSPACE;
+  if (!aligned16(ws)) return BL_ERR_ALIGN;
+  PackArgs a{W, wt, N, K, G, layout, alpha_in, W_packed, alpha, beta, rowsum, ws};
+  return launch_binarize_pack(a, (cudaStream_t)stream) == cudaSuccess ? BL_OK : BL_ERR_CUDA;
+}
+
+bl_status bitlinear_quant_act(const void* x, bl_dtype xt, int64_t M, int64_t K, int G, int b,
+                              bl_quant_mode mode, bl_gran gran, float ln_eps, int8_t* x_q,
+                              float* gamma, float* eta, void* ws, size_t ws_bytes, void* stream) {
+  if (!x || !x_q || !gamma) return BL_ERR_NULL;
+  if (mode == BL_ETA && !eta) return BL_ERR_NULL;
+  if (M <= 0) return BL_ERR_SHAPE;
+  bl_status st = check_kg(K, G);
+  if (st != BL_OK) return st;
+  if (b != 8 || !valid_dtype(xt)) return BL_ERR_UNSUPPORTED;
+  if (mode != BL_ABSMAX && mode != BL_ETA) return BL_ERR_UNSUPPORTED;
+  if (gran != BL_PER_TENSOR && gran != BL_PER_TOKEN) return BL_ERR_UNSUPPORTED;
+  if ((K / G) * sizeof(float) > 200 * 1024) return BL_ERR_SHAPE;   // one segment must fit in shared memory
+  if (M * (int64_t)G > 0x7FFFFFFF) return BL_ERR_SHAPE;
+  if (!aligned16(x) || !aligned16(x_q)) return BL_ERR_ALIGN;
+  if (gran == BL_PER_TENSOR) {
+    if (!ws || ws_bytes < bitlinear_workspace_bytes(BL_OP_QUANT_ACT, M, 1, K, G)) return BL_ERR_WORKSPACE;
+    if (!aligned16(ws)) return BL_ERR_ALIGN;
+  }
+  QuantArgs a{x, xt, M, K, G, mode, gran, ln_eps, x_q, gamma, eta, ws};
+  return launch_quant_act(a, (cudaStream_t)stream) == cudaSuccess ? BL_OK : BL_ERR_CUDA;
+}
+
+bl_status bitlinear_matmul_i32(const int8_t* x_q, int64_t M, int64_t K, int64_t N, int G,
+                               const uint8_t* W_packed, bl_layout layout, int32_t* acc, void* ws,
+                               size_t ws_bytes, void* stream) {
+  if (!x_q || !W_packed || !acc) return BL_ERR_NULL;
+  if (M <= 0 || N <= 0) return BL_ERR_SHAPE;
+  bl_status st = check_kg(K, G);
+  if (st != BL_OK) return st;
+  st = check_layout_for_gemm(layout, M, K, N, G);
+  if (st != BL_OK) return st;
+  if (!aligned16(x_q) || !aligned16(W_packed) || !aligned16(acc)) return BL_ERR_ALIGN;
+  if (!ws || ws_bytes < kStatusBytes) return BL_ERR_WORKSPACE;
+  if (!aligned16(ws)) return BL_ERR_ALIGN;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (cudaMemsetAsync(ws, 0, kStatusBytes, s) != cudaSuccess) return BL_ERR_CUDA;
+  GemmArgs a{};
+  a.x_q = x_q; a.M = M; a.K = K; a.N = N; a.G = G; a.W_packed = W_packed; a.acc = acc;
+  a.y = nullptr; a.gran = BL_PER_TENSOR; a.status = reinterpret_cast<uint32_t*>(ws);
+  cudaError_t e = (layout == BL_LAYOUT_PREFILL) ? launch_gemm_tc(a, s) : launch_gemm_simple(a, s);
+  return e == cudaSuccess ? BL_OK : BL_ERR_CUDA;
+}
+
+bl_status bitlinear_forward(const void* x, bl_dtype xt, int64_t M, int64_t K, int64_t N, int G,
+                            int b, bl_quant_mode mode, bl_gran gran, float ln_eps,
+                            int eta_correction, const uint8_t* W_packed, bl_layout layout,
+                            const float* beta, const int32_t* rowsum, void* y, bl_dtype yt,
+                            void* ws, size_t ws_bytes, void* stream) {
+  if (!x || !W_packed || !beta || !y) return BL_ERR_NULL;
+  if (eta_correction && !rowsum) return BL_ERR_NULL;
+  if (M <= 0 || N <= 0) return BL_ERR_SHAPE;
+  bl_status st = check_kg(K, G);
+  if (st != BL_OK) return st;
+  if (b != 8 || !valid_dtype(xt) || !valid_dtype(yt)) return BL_ERR_UNSUPPORTED;
+  if (mode != BL_ABSMAX && mode != BL_ETA) return BL_ERR_UNSUPPORTED;
+  if (gran != BL_PER_TENSOR && gran != BL_PER_TOKEN) return BL_ERR_UNSUPPORTED;
+  if (eta_correction && mode != BL_ETA) return BL_ERR_UNSUPPORTED;
+  st = check_layout_for_gemm(layout, M, K, N, G);
+  if (st != BL_OK) return st;
+  if ((K / G) * sizeof(float) > 200 * 1024 || M * (int64_t)G > 0x7FFFFFFF) return BL_ERR_SHAPE;
+  if (!aligned16(x) || !aligned16(W_packed) || !aligned16(y)) return BL_ERR_ALIGN;
+  const ForwardWs w = carve_forward(M, K, G);
+  if (!ws || ws_bytes < w.total) return BL_ERR_WORKSPACE;
+  if (!aligned16(ws)) return BL_ERR_ALIGN;
+  char* base = reinterpret_cast<char*>(ws);
+  cudaStream_t s = (cudaStream_t)stream;
+  if (cudaMemsetAsync(base + w.status, 0, kStatusBytes, s) != cudaSuccess) return BL_ERR_CUDA;
+  int8_t* codes = reinterpret_cast<int8_t*>(base + w.codes);
+  float* gamma = reinterpret_cast<float*>(base + w.gamma);
+  float* eta = reinterpret_cast<float*>(base + w.eta);
+  QuantArgs q{x, xt, M, K, G, mode, gran, ln_eps, codes, gamma, eta, base + w.quant};
+  if (launch_quant_act(q, s) != cudaSuccess) return BL_ERR_CUDA;
+  GemmArgs a{};
+  a.x_q = codes; a.M = M; a.K = K; a.N = N; a.G = G; a.W_packed = W_packed; a.acc = nullptr;
+  a.y = y; a.yt = yt; a.beta = beta; a.gamma = gamma; a.eta = eta; a.gran = gran;
+  a.rowsum = rowsum; a.eta_correction = eta_correction ? 1 : 0;
+  a.status = reinterpret_cast<uint32_t*>(base + w.status);
+  cudaError_t e = (layout == BL_LAYOUT_PREFILL) ? launch_gemm_tc(a, s) : launch_gemm_simple(a, s);
+  return e == cudaSuccess ? BL_OK : BL_ERR_CUDA;
+}
+
+bl_status bitlinear_gemv_decode(const void* x, bl_dtype xt, int64_t K, int64_t N, int G, int b,
+                                bl_quant_mode mode, float ln_eps, int eta_correction,
+                                const uint8_t* W_packed, const float* beta,
+                                const int32_t* rowsum, void* y, bl_dtype yt, void* stream) {
+  if (!x || !W_packed || !beta || !y) return BL_ERR_NULL;
+  if (eta_correction && !rowsum) return BL_ERR_NULL;
+  if (N <= 0) return BL_ERR_SHAPE;
+  bl_status st = check_kg(K, G);
+  if (st != BL_OK) return st;
+  if (b != 8 || !valid_dtype(xt) || !valid_dtype(yt)) return BL_ERR_UNSUPPORTED;
+  if (mode != BL_ABSMAX && mode != BL_ETA) return BL_ERR_UNSUPPORTED;
+  if (eta_correction && mode != BL_ETA) return BL_ERR_UNSUPPORTED;
+  if (K % 256 != 0 || N % 16 != 0 || K > 40960) return BL_ERR_SHAPE;
+  if (G > 1 && (K / G) % 128 != 0) return BL_ERR_SHAPE;
+  if (!aligned16(x) || !aligned16(W_packed) || !aligned16(y)) return BL_ERR_ALIGN;
+  GemvArgs a{x, xt, K, N, G, mode, ln_eps, eta_correction ? 1 : 0, W_packed, beta, rowsum, y, yt};
+  return launch_gemv_decode(a, (cudaStream_t)stream) == cudaSuccess ? BL_OK : BL_ERR_CUDA;
+}
+
+bl_status bitlinear_ws_status(const void* ws, void* stream) {
+  if (!ws) return BL_ERR_NULL;
+  uint32_t word = 0;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return BL_ERR_CUDA;
+  if (cudaMemcpy(&word, ws, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return BL_ERR_CUDA;
+  return word == 0 ? BL_OK : BL_ERR_TIMEOUT;
+}
+
+}  // extern "C"
