@@ -64,7 +64,7 @@ typedef enum { BL_PER_TENSOR = 0, BL_PER_TOKEN = 1 } bl_gran;
  *              every entry point except gemv_decode; shapes are unrestricted.
  *   PREFILL    the same bits re-tiled for the tensor-core GEMM: blocks of 128 rows x 128
  *              weights, rows and K padded up to multiples of 128 (see bitlinear_packed_bytes and
- *              bitlinear_layout_index).  Needs K % 16 == 0 and K_g % 128 == 0.
+ *              bitlinear_layout_index).  Needs K_g % 128 == 0.
  *   DECODE     the same bits re-ordered for the batch-1 GEMV.  Needs K % 256 == 0, N % 16 == 0. */
 typedef enum { BL_LAYOUT_CANONICAL = 0, BL_LAYOUT_PREFILL = 1, BL_LAYOUT_DECODE = 2 } bl_layout;
 
@@ -72,7 +72,8 @@ typedef enum {
   BL_OP_BINARIZE_PACK = 0,
   BL_OP_QUANT_ACT = 1,
   BL_OP_FORWARD = 2,
-  BL_OP_MATMUL_I32 = 3
+  BL_OP_MATMUL_I32 = 3,
+  BL_OP_MATMUL_DEQUANT = 4
 } bl_op;
 
 /* Human-readable name of a status code (static string, never NULL). */
@@ -135,6 +136,18 @@ bl_status bitlinear_forward(const void* x, bl_dtype xt, int64_t M, int64_t K, in
 bl_status bitlinear_matmul_i32(const int8_t* x_q, int64_t M, int64_t K, int64_t N, int G,
                                const uint8_t* W_packed, bl_layout layout, int32_t* acc, void* ws,
                                size_t ws_bytes, void* stream);
+
+/* Step 4 with the Eq. 11 rescale, for codes the caller already holds (the second half of
+ * bitlinear_forward; lets one LN+Quant of x feed several weight matrices, e.g. Q, K and V).
+ *   x_q [M,K] int8;  gamma, eta as written by bitlinear_quant_act for the same (mode, gran);
+ *   eta may be NULL unless eta_correction != 0.  Other arguments as for bitlinear_forward.
+ * The result is bit-identical to bitlinear_forward on the x that produced the codes.
+ * Workspace: BL_OP_MATMUL_DEQUANT. */
+bl_status bitlinear_matmul_dequant(const int8_t* x_q, int64_t M, int64_t K, int64_t N, int G,
+                                   bl_gran gran, const float* gamma, const float* eta,
+                                   int eta_correction, const uint8_t* W_packed, bl_layout layout,
+                                   const float* beta, const int32_t* rowsum, void* y, bl_dtype yt,
+                                   void* ws, size_t ws_bytes, void* stream);
 
 /* Steps 1, 2, 4 for one token (M = 1), fused in a single kernel that streams the packed
  * weights once; Eq. 11 with per-token gamma.  W_packed must be in DECODE layout.

@@ -18,13 +18,14 @@ F32, F16, BF16 = 0, 1, 2
 ABSMAX, ETA = 0, 1
 PER_TENSOR, PER_TOKEN = 0, 1
 CANONICAL, PREFILL, DECODE = 0, 1, 2
-OP_BINARIZE_PACK, OP_QUANT_ACT, OP_FORWARD, OP_MATMUL_I32 = 0, 1, 2, 3
+OP_BINARIZE_PACK, OP_QUANT_ACT, OP_FORWARD, OP_MATMUL_I32, OP_MATMUL_DEQUANT = 0, 1, 2, 3, 4
 MAX_GROUPS = 64
 
 EXPORTS = [
     "bitlinear_status_string", "bitlinear_workspace_bytes", "bitlinear_packed_bytes",
     "bitlinear_layout_index", "bitlinear_binarize_pack", "bitlinear_quant_act",
-    "bitlinear_forward", "bitlinear_matmul_i32", "bitlinear_gemv_decode", "bitlinear_ws_status",
+    "bitlinear_forward", "bitlinear_matmul_i32", "bitlinear_matmul_dequant", "bitlinear_gemv_decode",
+    "bitlinear_ws_status",
 ]
 
 _DTYPES = {torch.float32: F32, torch.float16: F16, torch.bfloat16: BF16}
@@ -63,6 +64,9 @@ def lib():
                                         vp, vp, vp, ci, vp, sz, vp]
         L.bitlinear_matmul_i32.restype = ci
         L.bitlinear_matmul_i32.argtypes = [vp, i64, i64, i64, ci, vp, ci, vp, vp, sz, vp]
+        L.bitlinear_matmul_dequant.restype = ci
+        L.bitlinear_matmul_dequant.argtypes = [vp, i64, i64, i64, ci, ci, vp, vp, ci, vp, ci, vp, vp, vp, ci,
+                                               vp, sz, vp]
         L.bitlinear_gemv_decode.restype = ci
         L.bitlinear_gemv_decode.argtypes = [vp, ci, i64, i64, ci, ci, ci, C.c_float, ci, vp, vp, vp,
                                             vp, ci, vp]
@@ -186,6 +190,21 @@ def matmul_i32(x_q, W_packed, N, G=1, layout=CANONICAL, acc=None, ws=None):
                                       ws.numel(), _stream())
     _check(code, "bitlinear_matmul_i32")
     return acc
+
+
+def matmul_dequant(x_q, gamma, W_packed, beta, N, G=1, gran=PER_TOKEN, layout=CANONICAL, eta=None,
+                   rowsum=None, eta_correction=False, out_dtype=torch.float32, y=None, ws=None):
+    """bitlinear_matmul_dequant.  x_q i8 [M,K] with its gamma (and eta); returns y [M,N]."""
+    M, K = x_q.shape
+    dev = x_q.device
+    if y is None:
+        y = torch.empty((M, N), dtype=out_dtype, device=dev)
+    ws = _ws(workspace_bytes(OP_MATMUL_DEQUANT, M, N, K, G), dev, ws)
+    code = lib().bitlinear_matmul_dequant(_ptr(x_q), M, K, N, G, gran, _ptr(gamma), _ptr(eta),
+                                          1 if eta_correction else 0, _ptr(W_packed), layout, _ptr(beta),
+                                          _ptr(rowsum), _ptr(y), _dt(y), _ptr(ws), ws.numel(), _stream())
+    _check(code, "bitlinear_matmul_dequant")
+    return y
 
 
 def gemv_decode(x, W_packed, beta, N, G=1, mode=ABSMAX, ln_eps=1e-5, rowsum=None,

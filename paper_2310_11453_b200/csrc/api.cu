@@ -20,13 +20,18 @@ inline bl_status check_kg(int64_t K, int G) {
 
 constexpr size_t kStatusBytes = 256;   // status word lives at the start of a GEMM workspace
 
+// A GEMM workspace is the status word followed by the tensor-core kernel's scratch.
+size_t gemm_ws_total(int64_t M, int64_t N, int G) {
+  return kStatusBytes + round256(gemm_tc_scratch_bytes(M, N, G));
+}
+
 struct ForwardWs {                     // carving of the BL_OP_FORWARD workspace
   size_t status, codes, gamma, eta, quant, total;
 };
-ForwardWs carve_forward(int64_t M, int64_t K, int G) {
+ForwardWs carve_forward(int64_t M, int64_t N, int64_t K, int G) {
   ForwardWs w;
   size_t off = 0;
-  w.status = off; off += kStatusBytes;
+  w.status = off; off += gemm_ws_total(M, N, G);
   w.codes = off;  off += round256((size_t)M * (size_t)K);
   w.gamma = off;  off += round256((size_t)M * (size_t)G * sizeof(float));
   w.eta = off;    off += round256((size_t)M * (size_t)G * sizeof(float));
@@ -60,13 +65,13 @@ const char* bitlinear_status_string(bl_status st) {
 }
 
 size_t bitlinear_workspace_bytes(bl_op op, int64_t M, int64_t N, int64_t K, int G) {
-  (void)N;
   if (check_kg(K, G) != BL_OK) return 0;
   switch (op) {
     case BL_OP_BINARIZE_PACK: return round256(pack_ws_bytes(G));
     case BL_OP_QUANT_ACT: return M > 0 ? round256(quant_ws_bytes(M, G)) : 0;
-    case BL_OP_FORWARD: return M > 0 ? carve_forward(M, K, G).total : 0;
-    case BL_OP_MATMUL_I32: return kStatusBytes;
+    case BL_OP_FORWARD: return (M > 0 && N > 0) ? carve_forward(M, N, K, G).total : 0;
+    case BL_OP_MATMUL_I32:
+    case BL_OP_MATMUL_DEQUANT: return (M > 0 && N > 0) ? gemm_ws_total(M, N, G) : 0;
   }
   return 0;
 }
@@ -146,13 +151,43 @@ bl_status bitlinear_matmul_i32(const int8_t* x_q, int64_t M, int64_t K, int64_t 
   st = check_layout_for_gemm(layout, M, K, N, G);
   if (st != BL_OK) return st;
   if (!aligned16(x_q) || !aligned16(W_packed) || !aligned16(acc)) return BL_ERR_ALIGN;
-  if (!ws || ws_bytes < kStatusBytes) return BL_ERR_WORKSPACE;
+  if (!ws || ws_bytes < gemm_ws_total(M, N, G)) return BL_ERR_WORKSPACE;
   if (!aligned16(ws)) return BL_ERR_ALIGN;
   cudaStream_t s = (cudaStream_t)stream;
   if (cudaMemsetAsync(ws, 0, kStatusBytes, s) != cudaSuccess) return BL_ERR_CUDA;
   GemmArgs a{};
   a.x_q = x_q; a.M = M; a.K = K; a.N = N; a.G = G; a.W_packed = W_packed; a.acc = acc;
   a.y = nullptr; a.gran = BL_PER_TENSOR; a.status = reinterpret_cast<uint32_t*>(ws);
+  a.scratch = reinterpret_cast<char*>(ws) + kStatusBytes;
+  cudaError_t e = (layout == BL_LAYOUT_PREFILL) ? launch_gemm_tc(a, s) : launch_gemm_simple(a, s);
+  return e == cudaSuccess ? BL_OK : BL_ERR_CUDA;
+}
+
+bl_status bitlinear_matmul_dequant(const int8_t* x_q, int64_t M, int64_t K, int64_t N, int G,
+                                   bl_gran gran, const float* gamma, const float* eta,
+                                   int eta_correction, const uint8_t* W_packed, bl_layout layout,
+                                   const float* beta, const int32_t* rowsum, void* y, bl_dtype yt,
+                                   void* ws, size_t ws_bytes, void* stream) {
+  if (!x_q || !W_packed || !beta || !gamma || !y) return BL_ERR_NULL;
+  if (eta_correction && (!rowsum || !eta)) return BL_ERR_NULL;
+  if (M <= 0 || N <= 0) return BL_ERR_SHAPE;
+  bl_status st = check_kg(K, G);
+  if (st != BL_OK) return st;
+  if (!valid_dtype(yt)) return BL_ERR_UNSUPPORTED;
+  if (gran != BL_PER_TENSOR && gran != BL_PER_TOKEN) return BL_ERR_UNSUPPORTED;
+  st = check_layout_for_gemm(layout, M, K, N, G);
+  if (st != BL_OK) return st;
+  if (!aligned16(x_q) || !aligned16(W_packed) || !aligned16(y)) return BL_ERR_ALIGN;
+  if (!ws || ws_bytes < gemm_ws_total(M, N, G)) return BL_ERR_WORKSPACE;
+  if (!aligned16(ws)) return BL_ERR_ALIGN;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (cudaMemsetAsync(ws, 0, kStatusBytes, s) != cudaSuccess) return BL_ERR_CUDA;
+  GemmArgs a{};
+  a.x_q = x_q; a.M = M; a.K = K; a.N = N; a.G = G; a.W_packed = W_packed; a.acc = nullptr;
+  a.y = y; a.yt = yt; a.beta = beta; a.gamma = gamma; a.eta = eta; a.gran = gran;
+  a.rowsum = rowsum; a.eta_correction = eta_correction ? 1 : 0;
+  a.status = reinterpret_cast<uint32_t*>(ws);
+  a.scratch = reinterpret_cast<char*>(ws) + kStatusBytes;
   cudaError_t e = (layout == BL_LAYOUT_PREFILL) ? launch_gemm_tc(a, s) : launch_gemm_simple(a, s);
   return e == cudaSuccess ? BL_OK : BL_ERR_CUDA;
 }
@@ -175,7 +210,7 @@ bl_status bitlinear_forward(const void* x, bl_dtype xt, int64_t M, int64_t K, in
   if (st != BL_OK) return st;
   if ((K / G) * sizeof(float) > 200 * 1024 || M * (int64_t)G > 0x7FFFFFFF) return BL_ERR_SHAPE;
   if (!aligned16(x) || !aligned16(W_packed) || !aligned16(y)) return BL_ERR_ALIGN;
-  const ForwardWs w = carve_forward(M, K, G);
+  const ForwardWs w = carve_forward(M, N, K, G);
   if (!ws || ws_bytes < w.total) return BL_ERR_WORKSPACE;
   if (!aligned16(ws)) return BL_ERR_ALIGN;
   char* base = reinterpret_cast<char*>(ws);
@@ -191,6 +226,7 @@ bl_status bitlinear_forward(const void* x, bl_dtype xt, int64_t M, int64_t K, in
   a.y = y; a.yt = yt; a.beta = beta; a.gamma = gamma; a.eta = eta; a.gran = gran;
   a.rowsum = rowsum; a.eta_correction = eta_correction ? 1 : 0;
   a.status = reinterpret_cast<uint32_t*>(base + w.status);
+  a.scratch = base + w.status + kStatusBytes;
   cudaError_t e = (layout == BL_LAYOUT_PREFILL) ? launch_gemm_tc(a, s) : launch_gemm_simple(a, s);
   return e == cudaSuccess ? BL_OK : BL_ERR_CUDA;
 }

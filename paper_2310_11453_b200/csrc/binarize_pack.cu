@@ -87,17 +87,7 @@ finalize_means(int64_t N, int64_t K, int G, int nblocks, const float* __restrict
 __device__ __forceinline__ uint32_t place_bits(uint32_t byte, int j, int layout) {
   if (layout == BL_LAYOUT_CANONICAL) return byte << (8 * j);
   uint32_t out = 0;
-  if (layout == BL_LAYOUT_PREFILL) {
-    // 16-weight chunks; weight q of a chunk sits at bit q/4 + 4*(q%4) of the chunk's u16.
-    const int qbase = (j & 1) * 8;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const int q = qbase + i;
-      out |= ((byte >> i) & 1u) << ((q >> 2) + 4 * (q & 3));
-    }
-    return out << (16 * (j >> 1));
-  }
-  // DECODE: weight q of the 32-weight word sits at bit q/4 + 8*(q%4).
+  // PREFILL and DECODE: weight q of the 32-weight word sits at bit q/4 + 8*(q%4).
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const int q = 8 * j + i;
@@ -202,9 +192,9 @@ int64_t prefill_bytes(int64_t N, int64_t K) {
 void prefill_index(int64_t K, int64_t n, int64_t k, int64_t* byte_off, int* bit) {
   const int64_t Kp = (K + 127) / 128 * 128;
   const int64_t block = (n >> 7) * (Kp >> 7) + (k >> 7);
-  const int chunk = (int)((k & 127) >> 4), q = (int)(k & 15);
-  const int p = (q >> 2) + 4 * (q & 3);
-  *byte_off = block * 2048 + (n & 127) * 16 + chunk * 2 + (p >> 3);
+  const int q = (int)(k & 31);
+  const int p = (q >> 2) + 8 * (q & 3);
+  *byte_off = block * 2048 + (n & 127) * 16 + ((k & 127) >> 5) * 4 + (p >> 3);
   *bit = p & 7;
 }
 

@@ -129,10 +129,12 @@ struct GemmArgs {
   const float* beta; const float* gamma; const float* eta; bl_gran gran;
   const int32_t* rowsum; int eta_correction;
   uint32_t* status;                                // device status word (tensor-core path)
+  void* scratch;                                   // gemm_tc_scratch_bytes(G) bytes (tensor-core path)
 };
 cudaError_t launch_gemm_simple(const GemmArgs& a, cudaStream_t s);
 cudaError_t launch_gemm_tc(const GemmArgs& a, cudaStream_t s);
 bool gemm_tc_supported(int64_t M, int64_t K, int64_t N, int G);
+size_t gemm_tc_scratch_bytes(int64_t M, int64_t N, int G);   // host-only, no device query
 
 struct GemvArgs {
   const void* x; bl_dtype xt; int64_t K, N; int G; bl_quant_mode mode; float ln_eps;

@@ -220,7 +220,7 @@ def test_matmul_i32_bit_exact(M, N, K, G):
         else:
             from tests.util import from_canonical
             packed = torch.from_numpy(from_canonical(bits.numpy(), layout, N, K)).to(DEV)
-        ws = torch.zeros(4096, dtype=torch.uint8, device=DEV)
+        ws = torch.zeros(B.workspace_bytes(B.OP_MATMUL_I32, M, N, K, G), dtype=torch.uint8, device=DEV)
         acc = B.matmul_i32(codes.to(DEV), packed, N, G=G, layout=layout, ws=ws)
         assert B.ws_status(ws) == B.OK
         assert (acc.cpu().numpy() == ref).all(), f"layout {layout}"
@@ -298,6 +298,22 @@ FORWARD_CASES = [
 def test_forward(M, K, N, G, dtype, ydtype, mode, gran, outliers, relu, seed):
     for layout in gemm_layouts(K, G):
         run_forward_case(M, K, N, G, dtype, ydtype, mode, gran, outliers, relu, seed, layout)
+
+
+def test_matmul_dequant_is_the_second_half_of_forward():
+    M, K, N, G = 150, 1024, 264, 2
+    x = synth.make_x(M, K, torch.bfloat16, seed=41, outliers=False, relu=True).to(DEV)
+    W = synth.make_w(N, K, torch.float32, seed=41).to(DEV)
+    for layout in gemm_layouts(K, G):
+        w = B.binarize_pack(W, G=G, layout=layout)
+        for gran in (B.PER_TENSOR, B.PER_TOKEN):
+            for corr in (False, True):
+                y = B.forward(x, w["W_packed"], w["beta"], N, G=G, mode=B.ETA, gran=gran, layout=layout,
+                              rowsum=w["rowsum"], eta_correction=corr, out_dtype=torch.float32)
+                q = B.quant_act(x, G=G, mode=B.ETA, gran=gran)
+                y2 = B.matmul_dequant(q["x_q"], q["gamma"], w["W_packed"], w["beta"], N, G=G, gran=gran,
+                                      layout=layout, eta=q["eta"], rowsum=w["rowsum"], eta_correction=corr)
+                assert torch.equal(y, y2)
 
 
 def test_forward_eta_correction():
