@@ -1,0 +1,447 @@
+#!/usr/bin/env python
+"""Benchmark of the BitLinear forward hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+One step = one BitLinear forward (LN + absmax quantisation, 1-bit x 8-bit matmul, rescale; Eq. 11)
+over the prefill batch: x bf16 [8192, 4096], W [4096, 4096] binarised and packed beforehand,
+per-tensor gamma, y bf16.  The headline value is the layer's integer throughput, 2*M*N*K / step
+time.  The same JSON line also carries the other rows of the path, each measured on its own
+workload: the batch-1 decode GEMV (K = 4096, N = 16384, 1000 calls in one CUDA graph rotating
+over 64 packed weight buffers), the LN+quant kernels and the binarise+pack kernels.
+
+Every rank runs the same replica on its own GPU (the layer has no exchange step); the job's
+value is the sum over ranks divided by the slowest rank's time.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "BitLinear prefill int8 TOPS + decode GEMV GB/s, % of B200 roofline"
+PREFILL = dict(M=8192, K=4096, N=4096, G=1)          # batch 4 x seq 2048, 6.7B-shaped projection
+DECODE = dict(K=4096, N=16384, calls=1000, buffers=64)
+ROTATE = 3                                           # distinct input/output sets per workload
+NOMINAL_INT8_TOPS = 4500.0
+NOMINAL_HBM_GBS = 8000.0
+INT8_TO_BF16 = 2.0                                   # nominal dense int8 : bf16 tensor rate
+
+
+def load_peaks():
+    """Measured denominators (copy bandwidth, bf16 GEMM) or the stated fallback."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index, period_s=0.002):
+        self.index, self.period, self.samples, self.reasons = index, period_s, [], set()
+        self.max_mhz, self._stop, self._thread, self._h, self._nv = None, threading.Event(), None, None, None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            uuid = torch.cuda.get_device_properties(index).uuid
+            try:
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + str(uuid)).encode())
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._nv = None
+
+    def _names(self, mask):
+        nv = self._nv
+        table = [("hw_slowdown", "nvmlClocksEventReasonHwSlowdown", 0x8),
+                 ("hw_thermal_slowdown", "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+                 ("sw_thermal_slowdown", "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+                 ("sw_power_cap", "nvmlClocksEventReasonSwPowerCap", 0x4),
+                 ("hw_power_brake", "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80)]
+        return {name for name, attr, default in table if mask & getattr(nv, attr, default)}
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                self.reasons |= self._names(mask)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return self._smi_once()
+        return dict(sm_mhz=statistics.median(self.samples), sm_max_mhz=self.max_mhz,
+                    reasons=sorted(self.reasons), samples=len(self.samples), source="nvml")
+
+    def _smi_once(self):
+        try:
+            out = subprocess.check_output(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=clocks.sm,clocks.max.sm",
+                 "--format=csv,noheader,nounits"], timeout=10).decode().split(",")
+            return dict(sm_mhz=float(out[0]), sm_max_mhz=float(out[1]), reasons=[], samples=1,
+                        source="nvidia-smi after the run")
+        except Exception:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0, source="unavailable")
+
+
+def event_pairs_ms(pairs):
+    return [a.elapsed_time(b) for a, b in pairs]
+
+
+# --------------------------------------------------------------------------------------- own arm
+
+def run_b200(args):
+    from paper_2310_11453_b200 import binding as B
+    from paper_2310_11453_b200 import synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the BitLinear library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+    B.lib()                                           # fail here, loudly, if the library is missing
+    peaks = load_peaks()
+    K_steps, W_steps = args.steps, max(args.warmup, 3)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if dist is None:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- prefill workload: inputs resident in HBM, ROTATE distinct sets (> L2 in total) ----------
+    M, K, N, G = PREFILL["M"], PREFILL["K"], PREFILL["N"], PREFILL["G"]
+    xs_host = [synth.make_x(M, K, torch.bfloat16, seed=2 + 101 * r + 7919 * rank, outliers=True).pin_memory()
+               for r in range(ROTATE)]
+    xs = [x.to(dev) for x in xs_host]
+    W = synth.make_w(N, K, torch.float32, seed=2).to(dev)
+    w = B.binarize_pack(W, G=G, layout=B.PREFILL)
+    ys = [torch.empty((M, N), dtype=torch.bfloat16, device=dev) for _ in range(ROTATE)]
+    qs = [dict(x_q=torch.empty((M, K), dtype=torch.int8, device=dev),
+               gamma=torch.empty(G, dtype=torch.float32, device=dev),
+               eta=torch.zeros(G, dtype=torch.float32, device=dev)) for _ in range(ROTATE)]
+    ws_q = torch.empty(B.workspace_bytes(B.OP_QUANT_ACT, M, 1, K, G), dtype=torch.uint8, device=dev)
+    ws_g = torch.empty(B.workspace_bytes(B.OP_MATMUL_DEQUANT, M, N, K, G), dtype=torch.uint8, device=dev)
+    ws_f = torch.empty(B.workspace_bytes(B.OP_FORWARD, M, N, K, G), dtype=torch.uint8, device=dev)
+
+    def step(i, ev=None):
+        r = i % ROTATE
+        if ev is not None:
+            ev[0].record()
+        B.quant_act(xs[r], G=G, mode=B.ABSMAX, gran=B.PER_TENSOR, out=qs[r], ws=ws_q)
+        if ev is not None:
+            ev[1].record()
+        B.matmul_dequant(qs[r]["x_q"], qs[r]["gamma"], w["W_packed"], w["beta"], N, G=G, gran=B.PER_TENSOR,
+                         layout=B.PREFILL, y=ys[r], ws=ws_g)
+        if ev is not None:
+            ev[2].record()
+
+    for i in range(W_steps):
+        step(i)
+    assert B.ws_status(ws_g) == B.OK, "tensor-core GEMM reported a device-side timeout"
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K_steps)]
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    with ClockSampler(local) as clocks:
+        t0.record()
+        for i in range(K_steps):
+            step(i, evs[i])
+        t1.record()
+        barrier()
+    total_ms = max_over_ranks(t0.elapsed_time(t1))
+    assert B.ws_status(ws_g) == B.OK
+    ms_per_step = total_ms / K_steps
+    ops_per_step = 2.0 * M * N * K
+    value = world * ops_per_step / (ms_per_step * 1e-3) / 1e12
+    gemm_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
+    quant_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
+    gemm_tops = ops_per_step / (gemm_ms * 1e-3) / 1e12
+    tensor_peak = INT8_TO_BF16 * peaks["bf16_tflops"]
+    quant_bytes = 2.0 * M * K * 2 + M * K                      # per-tensor: x read twice, codes written
+    quant_gbs = quant_bytes / (quant_ms * 1e-3) / 1e9
+
+    # ---- end to end through the public call, host buffers, copies inside the timed region -------
+    x_dev = torch.empty((M, K), dtype=torch.bfloat16, device=dev)
+    y_dev = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+    y_host = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+
+    def e2e_step(i):
+        x_dev.copy_(xs_host[i % ROTATE], non_blocking=True)
+        B.forward(x_dev, w["W_packed"], w["beta"], N, G=G, mode=B.ABSMAX, gran=B.PER_TENSOR,
+                  layout=B.PREFILL, y=y_dev, ws=ws_f)
+        y_host.copy_(y_dev, non_blocking=True)
+
+    e2e_steps = min(K_steps, 100)
+    for i in range(3):
+        e2e_step(i)
+    barrier()
+    t0.record()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    t1.record()
+    barrier()
+    e2e_ms = max_over_ranks(t0.elapsed_time(t1)) / e2e_steps
+    e2e = dict(value=world * ops_per_step / (e2e_ms * 1e-3) / 1e12, unit="TOPS", ms_per_step=e2e_ms,
+               h2d_bytes_per_step=M * K * 2, d2h_bytes_per_step=M * N * 2,
+               call="bitlinear_forward on device copies of pinned host x; y copied back to pinned host")
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": world, "steps": K_steps,
+        "warmup": W_steps, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8 x 1-bit -> int32, fp32 rescale", "data": "synthetic",
+        "config": {"workload": "prefill BitLinear forward: x bf16 [8192,4096] N(0,1) + 0.1% x20 outliers, "
+                               "W [4096,4096] N(0,0.02) binarised+packed beforehand, b=8, per-tensor gamma, "
+                               "y bf16",
+                   "M": M, "K": K, "N": N, "G": G, "parallelism": "replicas only" if world > 1 else "1 GPU",
+                   "l2": f"rotating over {ROTATE} input/output sets, {ROTATE * (M * K * 3 + M * N * 2) >> 20} MiB "
+                         "in total, larger than L2"},
+        "clocks": None,
+        "e2e": e2e,
+        "gpu_launches": 4 * K_steps,
+        "kernels_per_step": ["init_scope", "tensor_stats", "tensor_codes", "gemm_tc_kernel"],
+        "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": gemm_tops, "peak": tensor_peak,
+                     "unit": "TFLOP/s", "frac": gemm_tops / tensor_peak, "traffic": None,
+                     "op_kind": "int8 (s8 x s8 -> s32), 2 ops per multiply-accumulate",
+                     "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} x {INT8_TO_BF16} "
+                                    "(nominal int8:bf16 ratio)",
+                     "frac_of_nominal": gemm_tops / NOMINAL_INT8_TOPS, "avg_launch_ms": gemm_ms},
+        "roofline_quant": {"bound": "hbm", "kernel": "tensor_stats + tensor_codes", "achieved": quant_gbs,
+                           "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": quant_gbs / peaks["hbm_gbs"],
+                           "traffic": None, "avg_ms": quant_ms, "peak_source": peaks["source"] + " copy"},
+    }
+
+    parts = set(args.parts.split(","))
+    if rank == 0 and world == 1:
+        if "decode" in parts:
+            line["decode"] = bench_decode(B, synth, dev, peaks)
+        if "pack" in parts:
+            line["pack"] = bench_pack(B, synth, dev, peaks)
+        if "cpu" in parts:
+            line["cpu_baseline"] = cpu_baseline_prefill(xs_host[0], W.cpu())
+    line["clocks"] = clocks.summary()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def bench_decode(B, synth, dev, peaks):
+    """Batch-1 decode: 1000 GEMV calls in one CUDA graph, rotating over 64 packed weight buffers
+    (512 MiB, so every call streams its weights from HBM) with a fresh x per call."""
+    K, N, calls, nbuf = DECODE["K"], DECODE["N"], DECODE["calls"], DECODE["buffers"]
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(1)
+    packs = []
+    for _ in range(nbuf):
+        Wd = torch.randn((N, K), generator=gen, device=dev, dtype=torch.float32) * synth.W_STD
+        packs.append(B.binarize_pack(Wd, layout=B.DECODE, want_rowsum=False))
+        del Wd
+    x = synth.make_x(calls, K, torch.float16, seed=1, outliers=False).to(dev)
+    y = torch.empty((calls, N), dtype=torch.float16, device=dev)
+
+    def issue(n_bufs):
+        for i in range(calls):
+            p = packs[i % n_bufs]
+            B.gemv_decode(x[i], p["W_packed"], p["beta"], N, y=y[i])
+
+    issue(nbuf)
+    torch.cuda.synchronize()
+    out = {}
+    for name, n_bufs in (("hbm", nbuf), ("l2_hot", 1)):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            issue(n_bufs)
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        times = []
+        for _ in range(10):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            graph.replay()
+            b.record()
+            torch.cuda.synchronize()
+            times.append(a.elapsed_time(b))
+        out[name] = statistics.median(times) / calls * 1e3       # us per call
+        del graph
+    bytes_per_call = N * K / 8 + 2 * K + 2 * N
+    gbs = bytes_per_call / (out["hbm"] * 1e-6) / 1e9
+    return {"workload": "decode GEMV: x fp16 [1,4096], packed 1-bit W K=4096 N=16384, y fp16; 1000 calls in one "
+                        "CUDA graph over 64 weight buffers (512 MiB > L2), fresh x per call",
+            "us_per_call": out["hbm"], "us_per_call_l2_hot": out["l2_hot"], "bytes_per_call": bytes_per_call,
+            "gpu_launches": calls,
+            "roofline": {"bound": "hbm", "kernel": "gemv_decode_kernel", "achieved": gbs, "peak": peaks["hbm_gbs"],
+                         "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": None,
+                         "frac_of_nominal": gbs / NOMINAL_HBM_GBS, "peak_source": peaks["source"] + " copy"}}
+
+
+def bench_pack(B, synth, dev, peaks):
+    """Binarise+pack of the prefill weight matrix (fp32 [4096,4096]), rotating over 3 copies."""
+    N, K = PREFILL["N"], PREFILL["K"]
+    Ws = [synth.make_w(N, K, torch.float32, seed=2 + r).to(dev) for r in range(ROTATE)]
+    outs = [B.binarize_pack(Wr, layout=B.PREFILL) for Wr in Ws]
+    ws = torch.empty(B.workspace_bytes(B.OP_BINARIZE_PACK, 1, N, K, 1), dtype=torch.uint8, device=dev)
+    reps = 30
+    for i in range(3):
+        B.binarize_pack(Ws[i % ROTATE], layout=B.PREFILL, out=outs[i % ROTATE], ws=ws)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record()
+    for i in range(reps):
+        B.binarize_pack(Ws[i % ROTATE], layout=B.PREFILL, out=outs[i % ROTATE], ws=ws)
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / reps
+    nbytes = 2.0 * N * K * 4 + N * K / 8
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"workload": "binarize+pack W fp32 [4096,4096] -> 1 bit/weight (PREFILL layout), alpha, beta, rowsum",
+            "ms": ms, "gpu_launches": 3 * reps,
+            "roofline": {"bound": "hbm", "kernel": "reduce_partials + sign_pack", "achieved": gbs,
+                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": None,
+                         "peak_source": peaks["source"] + " copy"}}
+
+
+# --------------------------------------------------------------------------- the CPU oracle, timed
+
+def oracle_prefill_sample(x_host, W_host, tokens, reps=1):
+    """Times the CPU oracle's forward (LN+quant, matmul, rescale) on the first `tokens` tokens of the
+    prefill batch against the full weight matrix.  Returns (seconds per call, threads)."""
+    from oracle import oracle as O
+    xs = x_host[:tokens].to(torch.float32).numpy()
+    wb = O.binarize(W_host.numpy())
+    best = None
+    for _ in range(reps):
+        t = time.perf_counter()
+        O.forward(xs, wb["bits"], wb["beta"], G=1, mode=O.ABSMAX, gran=O.PER_TENSOR, ln_eps=1e-5)
+        dt = time.perf_counter() - t
+        best = dt if best is None else min(best, dt)
+    return best, O.num_threads()
+
+
+def cpu_baseline_prefill(x_host, W_host, target_s=15.0):
+    # two probes separate the fixed cost (unpacking W) from the per-token cost
+    d1, _ = oracle_prefill_sample(x_host, W_host, 64)
+    d2, _ = oracle_prefill_sample(x_host, W_host, 512)
+    per_token = max((d2 - d1) / 448.0, 1e-7)
+    tokens = int(min(PREFILL["M"], max(512, (target_s - d1) / per_token)))
+    tokens -= tokens % 64
+    dt, cores = oracle_prefill_sample(x_host, W_host, tokens)
+    ops = 2.0 * tokens * PREFILL["N"] * PREFILL["K"]
+    return {"value": ops / dt / 1e12, "unit": "TOPS", "cores": cores, "kind": "oracle",
+            "sample": f"oracle forward on the first {tokens} of {PREFILL['M']} tokens of the prefill batch, "
+                      f"full W [4096,4096]; {dt:.2f} s"}
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle as it stands, on the host cores, same metric and config.
+    Each step is the oracle's forward on a token sample of the prefill batch (16 to 1024 tokens,
+    sized so that the run ends in about a minute)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2310_11453_b200 import synth
+    M, K, N = PREFILL["M"], PREFILL["K"], PREFILL["N"]
+    from oracle import oracle as O
+    x_all = synth.make_x(1024, K, torch.bfloat16, seed=2, outliers=True)
+    W = synth.make_w(N, K, torch.float32, seed=2)
+    wb = O.binarize(W.numpy())
+    # size the per-step token sample so that the whole run takes about a minute
+    probe = x_all[:16].to(torch.float32).numpy()
+    t = time.perf_counter()
+    O.forward(probe, wb["bits"], wb["beta"], G=1, mode=O.ABSMAX, gran=O.PER_TENSOR, ln_eps=1e-5)
+    per_token = (time.perf_counter() - t) / 16
+    budget = 60.0 / (args.steps + max(args.warmup, 1))
+    tokens = int(max(16, min(1024, budget / max(per_token, 1e-9))))
+    tokens -= tokens % 16
+    xs = x_all[:tokens].to(torch.float32).numpy()
+
+    def step():
+        O.forward(xs, wb["bits"], wb["beta"], G=1, mode=O.ABSMAX, gran=O.PER_TENSOR, ln_eps=1e-5)
+
+    for _ in range(max(args.warmup, 1)):
+        step()
+    t = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t) / args.steps
+    value = 2.0 * tokens * N * K / dt / 1e12
+    sample = f"oracle forward on {tokens} of {M} tokens of the prefill batch per step, full W [4096,4096]"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "TOPS",
+            "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64 and exact integers (CPU oracle)", "data": "synthetic",
+            "config": {"workload": "prefill BitLinear forward (CPU oracle on a token sample)", "M": M, "K": K,
+                       "N": N, "G": 1, "sample_tokens": tokens},
+            "cpu_baseline": {"value": value, "unit": "TOPS", "cores": O.num_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--parts", default="decode,pack,cpu",
+                    help="extra measurements beside the prefill step (comma list of decode, pack, cpu; "
+                         "'none' for the prefill step alone, e.g. under a profiler)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_b200(args)
+
+
+if __name__ == "__main__":
+    main()
