@@ -10,8 +10,9 @@
 //   warp 1      MMA issuer (one thread): 4 MMAs of 128x256x32 per stage, tcgen05.commit
 //   warp 2      owns the tensor-memory allocation (512 columns = two 128x256 accumulators)
 //   warps 4-7   epilogue: tcgen05.ld one accumulator while the MMAs fill the other
-//   warps 8-15  weight expanders: thread u owns row u of the 256-row B tile; 16 bytes of bits
-//               come straight from global memory (prefetched two stages ahead in registers)
+//   warps 8-23  weight expanders in two groups of 8 warps that take alternate stages: thread u
+//               of a group owns row u of the 256-row B tile; its 16 bytes of bits come straight
+//               from global memory (prefetched two owned stages ahead in registers)
 // Stage hand-over uses mbarriers: full_a (TMA bytes), full_b (8 expander warps), empty
 // (tcgen05.commit), and a full/empty pair per accumulator.  Writes of the expanders are
 // generic-proxy stores, so each thread issues fence.proxy.async before its warp arrives.
@@ -39,7 +40,7 @@ constexpr int kBM = 128;                 // tokens per tile (MMA M, tensor-memor
 constexpr int kBN = 256;                 // output features per tile (MMA N)
 constexpr int kBK = 128;                 // weights per stage (one 128-byte swizzle atom)
 constexpr int kStages = 4;
-constexpr int kThreads = 512;
+constexpr int kThreads = 768;
 constexpr int kExpandWarp0 = 8;          // first expander warp
 constexpr int kEpiWarp0 = 4;             // first epilogue warp
 constexpr int kABytes = kBM * kBK;       // 16 KB
@@ -247,7 +248,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_byt
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&ctl->full_a[s]), 1);
-      mbar_init(smem_u32(&ctl->full_b[s]), kThreads / 32 - kExpandWarp0);
+      mbar_init(smem_u32(&ctl->full_b[s]), kBN / 32);
       mbar_init(smem_u32(&ctl->empty[s]), 1);
     }
     for (int b = 0; b < 2; ++b) {
@@ -325,15 +326,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_byt
     }
   } else if (warp >= kExpandWarp0) {
     // ---------------------------------------------------------------- weight expanders
-    const int u = threadIdx.x - kExpandWarp0 * 32;           // row of the B tile, 0..255
-    const uint32_t row_off = (uint32_t)u * 128u;
-    const uint32_t sw = (uint32_t)(u & 7);
-    int stage = 0; uint32_t phase = 0;
-    // flat walk over (tile, k-block) with a two-deep register prefetch of the 16 bytes of bits
+    // Two groups of 8 warps take alternate stages, so one group's stores, proxy fence and
+    // barrier round trip overlap the other group's arithmetic.
+    const int eg = (warp - kExpandWarp0) >> 3;                       // group 0 or 1
+    const int u = (threadIdx.x - kExpandWarp0 * 32) & (kBN - 1);     // row of the B tile, 0..255
+    // byte offset of chunk position 0 of row u inside a stage, pre-xored with the row's swizzle
+    const uint32_t row_base = smem_u32(smem) + (uint32_t)kABytes + (uint32_t)u * 128u + ((uint32_t)(u & 7) << 4);
+    int stage = eg; uint32_t phase = 0;
+    // flat walk over (tile, k-block); this group owns every second step.  The 16 bytes of
+    // bits of the next two owned steps are prefetched in registers.
     TileIter pf_it(tiles, m_tiles);
-    int pf_kb = 0;
-    const uint8_t* pf_src = nullptr;                         // row u of the tile's first k-block
+    int pf_kb = eg;
+    const uint8_t* pf_src = nullptr;                                 // row u of the tile's first k-block
     auto seek = [&]() {
+      while (pf_it.valid() && pf_kb >= k_blocks) { pf_kb -= k_blocks; pf_it.next(); }
       pf_src = nullptr;
       if (pf_it.valid()) {
         const int64_t nb = (int64_t)pf_it.n_tile() * 2 + (u >> 7);
@@ -345,32 +351,40 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_byt
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
       if (pf_it.valid()) {
         if (pf_src) v = __ldg(reinterpret_cast<const uint4*>(pf_src + (size_t)pf_kb * 2048));
-        if (++pf_kb == k_blocks) { pf_kb = 0; pf_it.next(); seek(); }
+        pf_kb += 2;
+        if (pf_kb >= k_blocks) seek();
       }
       return v;
     };
     uint4 b0 = fetch(), b1 = fetch();
-    bool ok = true;
-    for (TileIter it(tiles, m_tiles); ok && it.valid(); it.next()) {
-      for (int kb = 0; kb < k_blocks; ++kb) {
-        const uint4 cur = b0;
-        b0 = b1;
-        b1 = fetch();
-        if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
-        unsigned char* bt = smem + (size_t)stage * kStageBytes + kABytes + row_off;
-        const uint32_t words[4] = {cur.x, cur.y, cur.z, cur.w};
+    // number of steps this group owns: ceil((my_tiles * k_blocks - eg) / 2)
+    const uint32_t my_tiles = (tiles > blockIdx.x) ? (tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0u;
+    const uint64_t flat = (uint64_t)my_tiles * (uint64_t)k_blocks;
+    const uint64_t owned = flat > (uint64_t)eg ? (flat - eg + 1) / 2 : 0;
+    for (uint64_t i = 0; i < owned; ++i) {
+      const uint4 cur = b0;
+      b0 = b1;
+      b1 = fetch();
+      bool got = true;
+      if (lane == 0) got = mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag);
+      got = __shfl_sync(0xFFFFFFFFu, got, 0);
+      __syncwarp();
+      if (!got) break;
+      const uint32_t dst = row_base + (uint32_t)stage * (uint32_t)kStageBytes;
+      const uint32_t words[4] = {cur.x, cur.y, cur.z, cur.w};
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          const uint32_t wd = words[c >> 1];
-          const int j0 = (c & 1) * 4;
-          const uint4 o = make_uint4(signs4(wd, j0), signs4(wd, j0 + 1), signs4(wd, j0 + 2), signs4(wd, j0 + 3));
-          *reinterpret_cast<uint4*>(bt + (((uint32_t)c ^ sw) << 4)) = o;
-        }
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&ctl->full_b[stage]));
-        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+      for (int c = 0; c < 8; ++c) {
+        const uint32_t wd = words[c >> 1];
+        const int j0 = (c & 1) * 4;
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst ^ ((uint32_t)c << 4)),
+                     "r"(signs4(wd, j0)), "r"(signs4(wd, j0 + 1)), "r"(signs4(wd, j0 + 2)),
+                     "r"(signs4(wd, j0 + 3)) : "memory");
       }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&ctl->full_b[stage]));
+      stage += 2;
+      if (stage >= kStages) { stage -= kStages; phase ^= 1u; }
     }
   } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + 4) {
     // ---------------------------------------------------------------- epilogue
