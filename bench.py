@@ -287,18 +287,35 @@ def bench_decode(B, synth, dev, peaks):
     x = synth.make_x(calls, K, torch.float16, seed=1, outliers=False).to(dev)
     y = torch.empty((calls, N), dtype=torch.float16, device=dev)
 
-    def issue(n_bufs):
+    side = [torch.cuda.Stream(device=dev) for _ in range(3)]
+
+    def issue(n_bufs, n_streams=1):
+        """Issues the 1000 calls; with n_streams > 1 call i goes to stream i % n_streams, so calls on
+        different streams are independent of one another (each stream keeps its own order)."""
+        main = torch.cuda.current_stream()
+        lanes = [main] + side[:n_streams - 1]
+        if n_streams > 1:
+            fork = torch.cuda.Event()
+            fork.record(main)
+            for st in lanes[1:]:
+                st.wait_event(fork)
         for i in range(calls):
             p = packs[i % n_bufs]
-            B.gemv_decode(x[i], p["W_packed"], p["beta"], N, y=y[i])
+            with torch.cuda.stream(lanes[i % n_streams]):
+                B.gemv_decode(x[i], p["W_packed"], p["beta"], N, y=y[i])
+        for st in lanes[1:]:
+            join = torch.cuda.Event()
+            join.record(st)
+            main.wait_event(join)
 
     issue(nbuf)
     torch.cuda.synchronize()
     out = {}
-    for name, n_bufs in (("hbm", nbuf), ("l2_hot", 1)):
+    for name, n_bufs, n_streams in (("hbm", nbuf, 1), ("hbm_2streams", nbuf, 2), ("hbm_4streams", nbuf, 4),
+                                    ("l2_hot", 1, 1)):
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph):
-            issue(n_bufs)
+            issue(n_bufs, n_streams)
         for _ in range(3):
             graph.replay()
         torch.cuda.synchronize()
@@ -314,10 +331,22 @@ def bench_decode(B, synth, dev, peaks):
         del graph
     bytes_per_call = N * K / 8 + 2 * K + 2 * N
     gbs = bytes_per_call / (out["hbm"] * 1e-6) / 1e9
+
+    def rate(us):
+        return bytes_per_call / (us * 1e-6) / 1e9
+
     return {"workload": "decode GEMV: x fp16 [1,4096], packed 1-bit W K=4096 N=16384, y fp16; 1000 calls in one "
-                        "CUDA graph over 64 weight buffers (512 MiB > L2), fresh x per call",
+                        "CUDA graph over 64 weight buffers (512 MiB > L2), fresh x per call, one stream "
+                        "(every call ordered after the one before it)",
             "us_per_call": out["hbm"], "us_per_call_l2_hot": out["l2_hot"], "bytes_per_call": bytes_per_call,
             "gpu_launches": calls,
+            "independent_streams": {
+                "note": "same 1000 calls spread round-robin over 2 / 4 streams inside the graph: calls on "
+                        "different streams do not wait for one another",
+                "us_per_call_2": out["hbm_2streams"], "us_per_call_4": out["hbm_4streams"],
+                "gbs_2": rate(out["hbm_2streams"]), "gbs_4": rate(out["hbm_4streams"]),
+                "frac_2": rate(out["hbm_2streams"]) / peaks["hbm_gbs"],
+                "frac_4": rate(out["hbm_4streams"]) / peaks["hbm_gbs"]},
             "roofline": {"bound": "hbm", "kernel": "gemv_decode_kernel", "achieved": gbs, "peak": peaks["hbm_gbs"],
                          "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": None,
                          "frac_of_nominal": gbs / NOMINAL_HBM_GBS, "peak_source": peaks["source"] + " copy"}}

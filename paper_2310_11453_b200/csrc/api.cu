@@ -243,7 +243,7 @@ bl_status bitlinear_gemv_decode(const void* x, bl_dtype xt, int64_t K, int64_t N
   if (b != 8 || !valid_dtype(xt) || !valid_dtype(yt)) return BL_ERR_UNSUPPORTED;
   if (mode != BL_ABSMAX && mode != BL_ETA) return BL_ERR_UNSUPPORTED;
   if (eta_correction && mode != BL_ETA) return BL_ERR_UNSUPPORTED;
-  if (K % 256 != 0 || N % 16 != 0 || K > 40960) return BL_ERR_SHAPE;
+  if (K % 256 != 0 || N % 16 != 0 || K > 32768) return BL_ERR_SHAPE;
   if (G > 1 && (K / G) % 128 != 0) return BL_ERR_SHAPE;
   if (!aligned16(x) || !aligned16(W_packed) || !aligned16(y)) return BL_ERR_ALIGN;
   GemvArgs a{x, xt, K, N, G, mode, ln_eps, eta_correction ? 1 : 0, W_packed, beta, rowsum, y, yt};
