@@ -17,7 +17,8 @@
 //      eta (which do need 1/sqrt(Var + eps)) are only used by the final rescale;
 //   3. per row, each lane multiplies its 128-weight chunk with the 128 codes it keeps in
 //      registers: sum_k W~[n,k] x~[k] = 2 * sum_{bit=1} x~[k] - sum_k x~[k].  Rows come in
-//      batches of up to 7 per warp; the next batch is loaded while the current one is reduced.
+//      batches of up to 7 per warp; a row's register is reloaded with the next batch's row as
+//      soon as the row has been used.
 //
 // DECODE layout: row-major like CANONICAL, but inside every 32-weight word weight q sits at bit
 // q/4 + 8*(q%4).  Then word & (0x01010101 << j) holds weights 4j..4j+3 as bytes that are 0 or
@@ -30,14 +31,17 @@ namespace bl {
 
 namespace {
 
-constexpr int kGemvThreads = 256;
+#ifndef BL_GEMV_THREADS
+#define BL_GEMV_THREADS 256
+#endif
+constexpr int kGemvThreads = BL_GEMV_THREADS;
 constexpr int kGemvWarps = kGemvThreads / 32;
 constexpr int kBatchRows = 7;            // rows per warp and batch (two batches live in registers)
 constexpr int kSlice = 4096;             // weights per warp slice = 32 lanes x 128
 constexpr float kRoundMagic = 12582912.f;   // 1.5 * 2^23: x + magic - magic is rne(x) for |x| < 2^22
 
 struct GemvShared {
-  double s1[kGemvWarps], s2[kGemvWarps];
+  float s1[kGemvWarps], s2[kGemvWarps];
   float lo[kGemvWarps], hi[kGemvWarps];
   float gamma[BL_MAX_GROUPS];
   float eta[BL_MAX_GROUPS];
@@ -52,22 +56,25 @@ __device__ __forceinline__ int code_slot(int k) {
   return (k & ~(kSlice - 1)) | ((((k >> 4) & 7) * 32 + ((k >> 7) & 31)) << 4) | (k & 15);
 }
 
-// 1/sqrt(d) and 1/d in fp64 from the fp32 hardware approximations and two Newton steps each
-// (relative error of the seed 2^-22, then 2^-43, then below one fp64 ulp); arguments outside
-// the fp32 range take the exact routines.
-__device__ __forceinline__ double rsqrt_f64(double d) {
-  if (!(d > 1e-30 && d < 1e30)) return d > 0.0 ? 1.0 / sqrt(d) : 0.0;
-  double y = (double)rsqrtf((float)d);
-  y = y * (1.5 - 0.5 * d * y * y);
-  y = y * (1.5 - 0.5 * d * y * y);
-  return y;
-}
+// 1/d in fp64 from the fp32 reciprocal and one Newton step (relative error 2^-23, then about
+// 2^-45: a code can differ from exact arithmetic only within 1e-11 of a rounding tie);
+// arguments outside the fp32 range take the exact division.
 __device__ __forceinline__ double rcp_f64(double d) {
   if (!(d > 1e-30 && d < 1e30)) return 1.0 / d;
-  double y = (double)__frcp_rn((float)d);
-  y = y * (2.0 - d * y);
-  y = y * (2.0 - d * y);
-  return y;
+  const double y = (double)__frcp_rn((float)d);
+  return y * (2.0 - d * y);
+}
+// 1/sqrt(v) to fp32 accuracy (it only scales the output); exact routine outside the fp32 range.
+__device__ __forceinline__ float rsqrt_scale(double v) {
+  if (!(v > 1e-30 && v < 1e30)) return v > 0.0 ? (float)(1.0 / sqrt(v)) : 0.f;
+  const float f = (float)v;
+  float y = rsqrtf(f);
+  return y * (1.5f - 0.5f * f * y * y);
+}
+// The rare element whose fp32 image is too close to a rounding tie: redone in fp64.  Kept out of
+// line so that the common path carries no fp64 instructions.
+__device__ __noinline__ int code_slow_path(float x, double c, double span) {
+  return (int)rint(((double)x - c) * ((double)kQb / span));
 }
 
 // 128 * sum over this lane's chunk of bit * code, for one row.
@@ -111,23 +118,25 @@ __device__ __forceinline__ void warp_sum8(T (&v)[8], int lane) {
   v[0] += __shfl_xor_sync(0xFFFFFFFFu, v[0], 1);
 }
 
-// Moments of 8 raw values: fp32 inside the group of 8, fp64 across groups.
-__device__ __forceinline__ void accumulate8(const float (&v)[8], double& s1, double& s2, float& mn, float& mx) {
-  const float p1 = ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
+// Moments of 8 raw values.  Inside a warp the sums are fp32 (at most K/8 values per lane); the
+// eight warp totals are then combined in fp64.  The mean moves a code by about 1e-7 of a step
+// at worst this way, and the sum of squares only feeds the output scale.
+__device__ __forceinline__ void accumulate8(const float (&v)[8], float& s1, float& s2, float& mn, float& mx) {
+  s1 += ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
   float p2 = 0.f;
 #pragma unroll
   for (int i = 0; i < 8; ++i) { p2 = fmaf(v[i], v[i], p2); mn = fminf(mn, v[i]); mx = fmaxf(mx, v[i]); }
-  s1 += (double)p1;
-  s2 += (double)p2;
+  s2 += p2;
 }
 
 struct GemvGeom {            // decided on the host
   int rows_per_cta, rpw, nbatches, nslices, rowslots;
+  uint32_t inv_nslices, inv_group_chunks;   // ceil(2^16 / d): (v * inv) >> 16 == v / d for v < 256
   double inv_kg;
 };
 
 template <typename TX, typename TY>
-__global__ void __launch_bounds__(kGemvThreads, 2)
+__global__ void __launch_bounds__(kGemvThreads, kGemvThreads <= 256 ? 2 : 1)
 gemv_decode_kernel(GemvArgs a, GemvGeom geo) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __shared__ GemvShared sh;
@@ -152,7 +161,7 @@ gemv_decode_kernel(GemvArgs a, GemvGeom geo) {
 
   // ---- x first (the chain to the codes hangs on it), staged as fp32 ------------------------------
   const TX* x = reinterpret_cast<const TX*>(a.x);
-  double s1 = 0.0, s2 = 0.0;
+  float s1 = 0.f, s2 = 0.f;
   float mn = INFINITY, mx = -INFINITY;
   for (int k = threadIdx.x * 8; k < K; k += kGemvThreads * 8) {
     float v[8];
@@ -163,31 +172,31 @@ gemv_decode_kernel(GemvArgs a, GemvGeom geo) {
   }
 
   // ---- work split inside the CTA; first batch of rows: loads in flight during the prologue --------
-  const int slice = warp % nslices, rowslot = warp / nslices;   // warps that share a row / rows side by side
-  const int chunk = slice * 32 + lane;                          // 128-weight chunk of this lane
+  const int rowslot = (int)(((uint32_t)warp * geo.inv_nslices) >> 16);   // rows side by side
+  const int slice = warp - rowslot * nslices;                            // warps that share a row
+  const int chunk = slice * 32 + lane;                                   // 128-weight chunk of this lane
   const bool active = chunk * 128 < K && rowslot < rowslots;
-  const int my_group = active ? (chunk * 128) / Kg : 0;
+  const int my_group = active ? (int)(((uint32_t)chunk * geo.inv_group_chunks) >> 16) : 0;
   const float beta_mine = __ldg(a.beta + my_group);
   const uint8_t* wlane = a.W_packed + (int64_t)chunk * 16;
-  auto load_batch = [&](int b, uint4 (&dst)[kBatchRows]) {
-    const int64_t n0 = row_begin + ((int64_t)b * rowslots + rowslot) * rpw;
-    const int nrows = active ? (int)min((int64_t)rpw, row_end - n0) : 0;
-    const uint8_t* p = wlane + n0 * Kb;
-#pragma unroll
-    for (int r = 0; r < kBatchRows; ++r) {
-      dst[r] = make_uint4(0u, 0u, 0u, 0u);
-      if (r < nrows) dst[r] = __ldcs(reinterpret_cast<const uint4*>(p + (int64_t)r * Kb));
-    }
+  // Row r of batch b for this warp slot; rows past the end read as all-zero bits.
+  auto load_row = [&](int b, int r) -> uint4 {
+    const int64_t n = row_begin + ((int64_t)b * rowslots + rowslot) * rpw + r;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (active && r < rpw && b < nbatches && n < row_end)
+      v = __ldcs(reinterpret_cast<const uint4*>(wlane + n * Kb));
+    return v;
   };
-  uint4 cur[kBatchRows], nxt[kBatchRows];
-  load_batch(0, cur);
+  uint4 cur[kBatchRows];
+#pragma unroll
+  for (int r = 0; r < kBatchRows; ++r) cur[r] = load_row(0, r);
 
   // ---- steps 1-2 on the token: LN per group, gamma/eta, codes ------------------------------------
   __syncthreads();
   for (int g = 0; g < G; ++g) {
     const float* seg = xf + g * Kg;
     if (G > 1) {
-      s1 = 0.0; s2 = 0.0; mn = INFINITY; mx = -INFINITY;
+      s1 = 0.f; s2 = 0.f; mn = INFINITY; mx = -INFINITY;
       for (int k = threadIdx.x * 8; k < Kg; k += kGemvThreads * 8) {
         const float4 p = *reinterpret_cast<const float4*>(seg + k);
         const float4 q = *reinterpret_cast<const float4*>(seg + k + 4);
@@ -198,51 +207,74 @@ gemv_decode_kernel(GemvArgs a, GemvGeom geo) {
     s1 = warp_sum(s1); s2 = warp_sum(s2); mn = warp_min(mn); mx = warp_max(mx);
     if (lane == 0) { sh.s1[warp] = s1; sh.s2[warp] = s2; sh.lo[warp] = mn; sh.hi[warp] = mx; }
     __syncthreads();
-    const double t1 = ((sh.s1[0] + sh.s1[1]) + (sh.s1[2] + sh.s1[3])) + ((sh.s1[4] + sh.s1[5]) + (sh.s1[6] + sh.s1[7]));
+    double t1 = 0.0;
+#pragma unroll
+    for (int w = 0; w < kGemvWarps; w += 4)
+      t1 += ((double)sh.s1[w] + (double)sh.s1[w + 1]) + ((double)sh.s1[w + 2] + (double)sh.s1[w + 3]);
     float xlo = sh.lo[0], xhi = sh.hi[0];
 #pragma unroll
     for (int w = 1; w < kGemvWarps; ++w) { xlo = fminf(xlo, sh.lo[w]); xhi = fmaxf(xhi, sh.hi[w]); }
-    // location c and slope A of the code map (see the header)
+    // location c and slope A of the code map (see the header).  The fast path only needs fp32
+    // images of A and B = -c A (its error is covered by the tie window tau); the exact fp64
+    // values are rebuilt inside the slow path.
     const bool ln = a.ln_eps >= 0.f;
     const double mean = ln ? t1 * geo.inv_kg : 0.0;
-    const double dlo = (double)xlo - mean, dhi = (double)xhi - mean;
-    double c, span;
-    if (a.mode == BL_ABSMAX) { c = mean; span = fmax(fabs(dlo), fabs(dhi)); }
-    else { c = (double)xlo; span = (double)xhi - (double)xlo; }
+    const float mean_f = (float)mean;
+    const float cf = (a.mode == BL_ABSMAX) ? mean_f : xlo;
+    const float span_f = (a.mode == BL_ABSMAX) ? fmaxf(fabsf(xlo - mean_f), fabsf(xhi - mean_f)) : xhi - xlo;
     // a constant segment has gamma = 0 whatever eps is: all codes are 0
-    const double A64 = span > 0.0 ? (double)kQb * rcp_f64(span) : 0.0;
-    const float Af = (float)A64, Bf = (float)(-c * A64);
-    const float tau = 4e-7f * (fabsf(Af) * fmaxf(fabsf(xlo), fabsf(xhi)) + fabsf(Bf) + 1.0f);
+    float Af = 0.f;
+    if (span_f > 0.f) {
+      const float y = __frcp_rn(span_f);
+      Af = (float)kQb * (y * (2.f - span_f * y));
+    }
+    const float Bf = -cf * Af;
+    const float tau = 1e-6f * (fabsf(Af) * fmaxf(fabsf(xlo), fabsf(xhi)) + fabsf(Bf) + 1.0f);
     const int code_lo = (a.mode == BL_ABSMAX) ? -kCodeMax : 0;
     for (int k = threadIdx.x * 8; k < Kg; k += kGemvThreads * 8) {
       const float4 p = *reinterpret_cast<const float4*>(seg + k);
       const float4 q = *reinterpret_cast<const float4*>(seg + k + 4);
       const float v[8] = {p.x, p.y, p.z, p.w, q.x, q.y, q.z, q.w};
-      uint32_t wq[2] = {0u, 0u};
+      int code[8];
+      bool near_tie = false;
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const float f = fmaf(v[i], Af, Bf);
         const float t = f + kRoundMagic;                               // rne(f) in the low mantissa bits
         const float r = t - kRoundMagic;
-        int code = __float_as_int(t) - __float_as_int(kRoundMagic);
-        if (fabsf(fabsf(f - r) - 0.5f) < tau)                          // too close to a tie for fp32
-          code = (int)rint(((double)v[i] - c) * A64);
-        code = max(code_lo, min(kCodeMax, code));
-        wq[i >> 2] |= (uint32_t)(code & 0xFF) << (8 * (i & 3));
+        code[i] = __float_as_int(t) - __float_as_int(kRoundMagic);
+        near_tie |= fabsf(fabsf(f - r) - 0.5f) < tau;
       }
+      if (near_tie && span_f > 0.f) {                                  // rare: redo the 8 codes exactly
+        const double c = (a.mode == BL_ABSMAX) ? mean : (double)xlo;
+        const double span = (a.mode == BL_ABSMAX) ? fmax(fabs((double)xlo - mean), fabs((double)xhi - mean))
+                                                  : (double)xhi - (double)xlo;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) code[i] = code_slow_path(v[i], c, span);
+      }
+      uint32_t wq[2] = {0u, 0u};
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        wq[i >> 2] |= (uint32_t)(max(code_lo, min(kCodeMax, code[i])) & 0xFF) << (8 * (i & 3));
       *reinterpret_cast<uint2*>(codes + code_slot(g * Kg + k)) = make_uint2(wq[0], wq[1]);
     }
     if (threadIdx.x == 0) {
-      // gamma and eta of Eq. 5 / 6 on x^ = (x - mean) rstd; only the final rescale reads them
-      const double t2 = ((sh.s2[0] + sh.s2[1]) + (sh.s2[2] + sh.s2[3])) + ((sh.s2[4] + sh.s2[5]) + (sh.s2[6] + sh.s2[7]));
-      double rstd = 1.0;
+      // gamma and eta of Eq. 5 / 6 on x^ = (x - mean) rstd; only the final rescale reads them,
+      // so fp32 is enough unless the mean dwarfs the spread (then the variance is formed in fp64)
+      float t2 = 0.f;
+#pragma unroll
+      for (int w = 0; w < kGemvWarps; w += 4) t2 += (sh.s2[w] + sh.s2[w + 1]) + (sh.s2[w + 2] + sh.s2[w + 3]);
+      float rstd = 1.f;
       if (ln) {
-        double var = t2 * geo.inv_kg - mean * mean;
+        const float inv_f = (float)geo.inv_kg;
+        float var_f = fmaf(-mean_f, mean_f, t2 * inv_f);
+        double var = (double)var_f;
+        if (!(mean_f * mean_f <= 16.f * var_f)) var = (double)t2 * geo.inv_kg - mean * mean;
         if (var < 0.0) var = 0.0;
-        rstd = rsqrt_f64(var + (double)a.ln_eps);
+        rstd = rsqrt_scale(var + (double)a.ln_eps);
       }
-      sh.gamma[g] = (float)(span * rstd);
-      sh.eta[g] = (a.mode == BL_ABSMAX) ? 0.f : (float)(dlo * rstd);
+      sh.gamma[g] = span_f * rstd;
+      sh.eta[g] = (a.mode == BL_ABSMAX) ? 0.f : (xlo - mean_f) * rstd;
     }
     __syncthreads();                                   // codes and gamma of g visible; sh.s1.. reusable
   }
@@ -270,20 +302,25 @@ gemv_decode_kernel(GemvArgs a, GemvGeom geo) {
   // ---- stream the rows of this CTA, one batch of rpw rows per warp at a time -------------------------
   TY* y = reinterpret_cast<TY*>(a.y);
   for (int b = 0; b < nbatches; ++b) {
-    if (b + 1 < nbatches) load_batch(b + 1, nxt);
+    // each row's register is refilled with the same row of the next batch as soon as it is used
     float (&part)[kGemvWarps][8] = sh.partial[b & 1];
     if (G == 1) {
       int v[8];
 #pragma unroll
-      for (int r = 0; r < kBatchRows; ++r) v[r] = active ? (chunk_dot128(cur[r], xr) >> 6) - csum : 0;   // Eq. 7: 2 S - sum x~
+      for (int r = 0; r < kBatchRows; ++r) {
+        v[r] = active ? (chunk_dot128(cur[r], xr) >> 6) - csum : 0;   // Eq. 7: 2 S - sum x~
+        cur[r] = load_row(b + 1, r);
+      }
       v[7] = 0;
       warp_sum8(v, lane);
       if ((lane & 3) == 0) part[warp][lane >> 2] = (float)v[0] * lane_scale;   // one group: the scale is uniform
     } else {
       float v[8];
 #pragma unroll
-      for (int r = 0; r < kBatchRows; ++r)
+      for (int r = 0; r < kBatchRows; ++r) {
         v[r] = active ? (float)((chunk_dot128(cur[r], xr) >> 6) - csum) * lane_scale : 0.f;
+        cur[r] = load_row(b + 1, r);
+      }
       v[7] = 0.f;
       warp_sum8(v, lane);
       if ((lane & 3) == 0) part[warp][lane >> 2] = v[0];
@@ -301,10 +338,6 @@ gemv_decode_kernel(GemvArgs a, GemvGeom geo) {
         }
         y[n] = out_cast<TY>(v);
       }
-    }
-    if (b + 1 < nbatches) {
-#pragma unroll
-      for (int r = 0; r < kBatchRows; ++r) cur[r] = nxt[r];
     }
   }
 }
@@ -326,6 +359,9 @@ cudaError_t run2(const GemvArgs& a, cudaStream_t s) {
   geo.nbatches = (int)nbatches;
   geo.rpw = (int)((per_slot + nbatches - 1) / nbatches);
   geo.inv_kg = 1.0 / (double)(a.K / a.G);
+  geo.inv_nslices = (65536u + geo.nslices - 1) / geo.nslices;
+  const uint32_t group_chunks = a.G > 1 ? (uint32_t)(a.K / a.G / 128) : 256u;   // G > 1 needs K_g % 128 == 0
+  geo.inv_group_chunks = (65536u + group_chunks - 1) / group_chunks;
   const unsigned grid = (unsigned)((a.N + rows_per_cta - 1) / rows_per_cta);
   const size_t smem = (size_t)a.K * sizeof(float) + (size_t)geo.nslices * kSlice;
   if (smem > 48 * 1024) {
