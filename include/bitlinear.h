@@ -47,7 +47,8 @@ typedef enum {
   BL_ERR_UNSUPPORTED = 4, /* b != 8, unknown enum value, or layout not accepted by this call */
   BL_ERR_WORKSPACE = 5,   /* ws is NULL or smaller than bitlinear_workspace_bytes() */
   BL_ERR_CUDA = 6,        /* a CUDA runtime call (launch, attribute, tensor map) failed */
-  BL_ERR_TIMEOUT = 7      /* a bounded device-side wait expired (read via bitlinear_ws_status) */
+  BL_ERR_TIMEOUT = 7,     /* a bounded device-side wait expired (read via bitlinear_ws_status) */
+  BL_ERR_TOO_LARGE = 8    /* the problem exceeds the built-in scratch of a *_noalloc entry point */
 } bl_status;
 
 typedef enum { BL_F32 = 0, BL_F16 = 1, BL_BF16 = 2 } bl_dtype;
@@ -115,6 +116,33 @@ bl_status bitlinear_binarize_pack(const void* W, bl_dtype wt, int64_t N, int64_t
 bl_status bitlinear_quant_act(const void* x, bl_dtype xt, int64_t M, int64_t K, int G, int b,
                               bl_quant_mode mode, bl_gran gran, float ln_eps, int8_t* x_q,
                               float* gamma, float* eta, void* ws, size_t ws_bytes, void* stream);
+
+/* bitlinear_quant_act for callers that cannot provide a workspace.  (The paper has no counterpart:
+ * this is a packaging variant of the entry point above, not another operation.)
+ *
+ * Who needs it: code that runs where device memory may not be allocated or sized at run time -
+ * a plug-in called from inside another framework's stream callback or graph-building phase, a
+ * real-time loop with a fixed memory budget, a host binding that only forwards pointers it was
+ * given.  Such callers still own x, x_q, gamma and eta, but have nowhere to put the statistics
+ * that the per-tensor path keeps between its two passes.
+ *
+ * The statistics go to a fixed array inside the library instead (about
+ * 24 * BL_NOALLOC_MAX_SEGMENTS bytes, resident on every GPU that loads the library until the
+ * process ends).  Consequences:
+ *   - BL_PER_TENSOR calls with M * G > BL_NOALLOC_MAX_SEGMENTS return BL_ERR_TOO_LARGE and launch
+ *     nothing.  BL_PER_TOKEN calls need no scratch and have no such limit.
+ *   - All calls on one GPU share the array.  Calls that may overlap on the GPU (different
+ *     streams) race on it and corrupt each other; keep them on one stream or order them yourself.
+ *     A call leaves nothing behind that the next one depends on.
+ *   - The first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress); make that first call outside any stream capture.
+ *   - No cudaMalloc, cudaFree or other allocating routine is called, now or later.
+ * Arguments, results, error codes and rounding are otherwise exactly those of bitlinear_quant_act;
+ * the same kernels run, so the outputs are bit-identical. */
+#define BL_NOALLOC_MAX_SEGMENTS 16384
+bl_status bitlinear_quant_act_noalloc(const void* x, bl_dtype xt, int64_t M, int64_t K, int G, int b,
+                                      bl_quant_mode mode, bl_gran gran, float ln_eps, int8_t* x_q,
+                                      float* gamma, float* eta, void* stream);
 
 /* Steps 1, 2, 4, Eq. 11: y = (W~ x~) . beta_g gamma / Q_b summed over groups in ascending order.
  *   eta_correction != 0 (BL_ETA only) adds eta.beta_g.rowsum[n,g], which undoes the shift of

@@ -20,10 +20,12 @@ PER_TENSOR, PER_TOKEN = 0, 1
 CANONICAL, PREFILL, DECODE = 0, 1, 2
 OP_BINARIZE_PACK, OP_QUANT_ACT, OP_FORWARD, OP_MATMUL_I32, OP_MATMUL_DEQUANT = 0, 1, 2, 3, 4
 MAX_GROUPS = 64
+NOALLOC_MAX_SEGMENTS = 16384
+ERR_TOO_LARGE = 8
 
 EXPORTS = [
     "bitlinear_status_string", "bitlinear_workspace_bytes", "bitlinear_packed_bytes",
-    "bitlinear_layout_index", "bitlinear_binarize_pack", "bitlinear_quant_act",
+    "bitlinear_layout_index", "bitlinear_binarize_pack", "bitlinear_quant_act", "bitlinear_quant_act_noalloc",
     "bitlinear_forward", "bitlinear_matmul_i32", "bitlinear_matmul_dequant", "bitlinear_gemv_decode",
     "bitlinear_ws_status",
 ]
@@ -59,6 +61,8 @@ def lib():
         L.bitlinear_binarize_pack.argtypes = [vp, ci, i64, i64, ci, ci, vp, vp, vp, vp, vp, vp, sz, vp]
         L.bitlinear_quant_act.restype = ci
         L.bitlinear_quant_act.argtypes = [vp, ci, i64, i64, ci, ci, ci, ci, C.c_float, vp, vp, vp, vp, sz, vp]
+        L.bitlinear_quant_act_noalloc.restype = ci
+        L.bitlinear_quant_act_noalloc.argtypes = [vp, ci, i64, i64, ci, ci, ci, ci, C.c_float, vp, vp, vp, vp]
         L.bitlinear_forward.restype = ci
         L.bitlinear_forward.argtypes = [vp, ci, i64, i64, i64, ci, ci, ci, ci, C.c_float, ci, vp, ci,
                                         vp, vp, vp, ci, vp, sz, vp]
@@ -162,6 +166,18 @@ def quant_act(x, G=1, mode=ABSMAX, gran=PER_TOKEN, ln_eps=1e-5, b=8, out=None, w
                                      _ptr(gamma), _ptr(eta), _ptr(ws), ws.numel(), _stream())
     _check(code, "bitlinear_quant_act")
     return dict(x_q=x_q, gamma=gamma, eta=eta)
+
+
+def quant_act_noalloc(x, G=1, mode=ABSMAX, gran=PER_TOKEN, ln_eps=1e-5, b=8, out=None):
+    """bitlinear_quant_act_noalloc: bitlinear_quant_act without a caller workspace (the per-tensor
+    statistics go to a fixed array inside the library).  `out` must carry x_q, gamma and eta: this
+    wrapper allocates nothing either.  Returns `out`."""
+    M, K = x.shape
+    code = lib().bitlinear_quant_act_noalloc(_ptr(x), _dt(x), M, K, G, b, mode, gran, float(ln_eps),
+                                             _ptr(out["x_q"]), _ptr(out["gamma"]), _ptr(out.get("eta")),
+                                             _stream())
+    _check(code, "bitlinear_quant_act_noalloc")
+    return out
 
 
 def forward(x, W_packed, beta, N, G=1, mode=ABSMAX, gran=PER_TOKEN, ln_eps=1e-5, layout=CANONICAL,

@@ -60,6 +60,7 @@ const char* bitlinear_status_string(bl_status st) {
     case BL_ERR_WORKSPACE: return "workspace missing or too small";
     case BL_ERR_CUDA: return "CUDA runtime error";
     case BL_ERR_TIMEOUT: return "device-side wait timed out";
+    case BL_ERR_TOO_LARGE: return "problem exceeds the built-in scratch of the no-allocation entry point";
   }
   return "unknown status";
 }

@@ -8,6 +8,8 @@
 // Per-tensor scope splits in two kernels: the first leaves each segment's moments in the
 // workspace and folds the extremes of x^ into a global atomic min/max on an order-preserving
 // encoding (order-independent, hence deterministic); the second re-reads x and writes codes.
+#include <mutex>
+
 #include "quant_core.cuh"
 
 namespace bl {
@@ -152,6 +154,34 @@ size_t quant_ws_bytes(int64_t M, int G) {
   return sizeof(TensorScope) + (size_t)M * (size_t)G * sizeof(SegRecord);
 }
 
+// ---- built-in scratch of bitlinear_quant_act_noalloc -------------------------------------------
+// Room for the per-tensor statistics of up to BL_NOALLOC_MAX_SEGMENTS (token, group) segments.
+// The array lives in the library image: every GPU that loads the library holds these bytes until
+// the process exits.  Host code must not hand the symbol itself to a kernel (on the host the name
+// is only a stand-in); it asks the runtime for the device address once per device.
+constexpr size_t kNoAllocBytes = sizeof(TensorScope) + (size_t)BL_NOALLOC_MAX_SEGMENTS * sizeof(SegRecord);
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
+
+// Device address of the built-in scratch on the current device (cached per device ordinal).
+static cudaError_t noalloc_scratch_address(void** out) {
+  constexpr int kMaxDevices = 64;
+  static void* cached[kMaxDevices] = {};
+  static std::mutex guard;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(guard);
+  if (cached[dev] == nullptr) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+    if (e != cudaSuccess) return e;
+    cached[dev] = p;
+  }
+  *out = cached[dev];
+  return cudaSuccess;
+}
+
 cudaError_t launch_quant_act(const QuantArgs& a, cudaStream_t s) {
   switch (a.xt) {
     case BL_F32: return run<float>(a, s);
@@ -162,3 +192,19 @@ cudaError_t launch_quant_act(const QuantArgs& a, cudaStream_t s) {
 }
 
 }  // namespace bl
+
+extern "C" bl_status bitlinear_quant_act_noalloc(const void* x, bl_dtype xt, int64_t M, int64_t K, int G, int b,
+                                                 bl_quant_mode mode, bl_gran gran, float ln_eps, int8_t* x_q,
+                                                 float* gamma, float* eta, void* stream) {
+  // Refuse what the built-in scratch cannot hold before anything else is looked at.
+  if (M > 0 && G > 0 && gran == BL_PER_TENSOR && M * (int64_t)G > (int64_t)BL_NOALLOC_MAX_SEGMENTS)
+    return BL_ERR_TOO_LARGE;
+  void* scratch = nullptr;
+  if (bl::noalloc_scratch_address(&scratch) != cudaSuccess) return BL_ERR_CUDA;
+  // Same validation and the same kernels as bitlinear_quant_act, with the scratch passed as its
+  // workspace.  tensor_stats rewrites every record it later reads and init_scope resets the
+  // running extremes, so nothing of an earlier call survives into this one.
+  return bitlinear_quant_act(x, xt, M, K, G, b, mode, gran, ln_eps, x_q, gamma, eta, scratch,
+                             bl::kNoAllocBytes, stream);
+}
+
