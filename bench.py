@@ -246,14 +246,14 @@ def run_b200(args):
         "clocks": None,
         "e2e": e2e,
         "gpu_launches": 4 * K_steps,
-        "kernels_per_step": ["init_scope", "tensor_stats", "tensor_codes", "gemm_tc_kernel"],
+        "kernels_per_step": ["init_scope", "rows_tensor_stats", "rows_tensor_codes", "gemm_tc_kernel"],
         "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": gemm_tops, "peak": tensor_peak,
                      "unit": "TFLOP/s", "frac": gemm_tops / tensor_peak, "traffic": None,
                      "op_kind": "int8 (s8 x s8 -> s32), 2 ops per multiply-accumulate",
                      "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} x {INT8_TO_BF16} "
                                     "(nominal int8:bf16 ratio)",
                      "frac_of_nominal": gemm_tops / NOMINAL_INT8_TOPS, "avg_launch_ms": gemm_ms},
-        "roofline_quant": {"bound": "hbm", "kernel": "tensor_stats + tensor_codes", "achieved": quant_gbs,
+        "roofline_quant": {"bound": "hbm", "kernel": "rows_tensor_stats + rows_tensor_codes", "achieved": quant_gbs,
                            "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": quant_gbs / peaks["hbm_gbs"],
                            "traffic": None, "avg_ms": quant_ms, "peak_source": peaks["source"] + " copy"},
     }

@@ -2,7 +2,9 @@
 // quantisation (Eq. 4-6, 14).  HBM-bound: x is read once (per token) or twice (per tensor) with
 // 128-bit loads; the normalised row is never written to HBM.
 //
-// One CTA per (token m, group g) segment of K_g features, staged in shared memory as fp32:
+// Two implementations.  Segments of up to 4096 16-bit (2048 fp32) features take the fast path in
+// the second half of this file: one warp per segment, the segment in registers.  Longer segments
+// take one CTA per (token m, group g) segment, staged in shared memory as fp32:
 //   moments  sum, raw min/max, then sum of squared deviations      (quant_core.cuh)
 //   codes    one FMA + round per element, 8 codes per 8-byte store
 // Per-tensor scope splits in two kernels: the first leaves each segment's moments in the
@@ -120,6 +122,245 @@ tensor_codes(const T* __restrict__ x, int64_t K, int G, int mode, const TensorSc
   }
 }
 
+
+// ================================================================================================
+// Fast path: one warp per (token, group) segment, the whole segment held in registers.
+//
+// Used when a segment fits 16 x 16 bytes per lane (K_g <= 4096 for 16-bit inputs, <= 2048 for
+// fp32), which covers every shape of the paper's model table.  A warp issues all loads of its
+// segment at once (up to 8 KB in flight per warp, 16 warps per SM), then takes the two LN passes
+// and the quantisation out of registers with warp shuffles only: no shared memory, no block
+// barrier.  Sums are fp32 inside a lane and fp64 across lanes; the second pass sums squared
+// deviations from the fp32-rounded mean and corrects for that rounding exactly.  Reciprocals and
+// the inverse square root are hardware seeds refined by Newton steps in fp64 (below one ulp of
+// fp64 after two steps), which keeps fp64 division and square-root routines out of the kernels.
+constexpr int kRowWarps = 8;
+constexpr int kRowRegs = 16;                                  // uint4 per lane
+constexpr float kRoundMagic = 12582912.f;                     // 1.5 * 2^23: x + magic - magic = rne(x), |x| < 2^22
+
+template <typename T> struct RowTraits {                      // chunk = 8 consecutive elements
+  static constexpr int kVecPerChunk = sizeof(T) == 4 ? 2 : 1;
+  static constexpr int kChunks = kRowRegs / kVecPerChunk;     // chunks per lane
+  static constexpr int kMaxKg = kChunks * 32 * 8;
+};
+
+__device__ __forceinline__ double rcp_newton(double d) {      // d > 0
+  if (!(d > 1e-30 && d < 1e30)) return 1.0 / d;
+  double y = (double)__frcp_rn((float)d);
+  y = y * (2.0 - d * y);
+  return y * (2.0 - d * y);
+}
+__device__ __forceinline__ double rsqrt_newton(double d) {    // d >= 0
+  if (!(d > 1e-30 && d < 1e30)) return d > 0.0 ? 1.0 / sqrt(d) : 0.0;
+  double y = (double)rsqrtf((float)d);
+  y = y * (1.5 - 0.5 * d * y * y);
+  return y * (1.5 - 0.5 * d * y * y);
+}
+
+template <typename T>
+__device__ __forceinline__ void row_load(const T* __restrict__ src, int nchunks, int lane, uint4 (&raw)[kRowRegs]) {
+  constexpr int V = RowTraits<T>::kVecPerChunk;
+#pragma unroll
+  for (int i = 0; i < RowTraits<T>::kChunks; ++i) {
+    const int c = lane + 32 * i;
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      raw[i * V + j] = make_uint4(0u, 0u, 0u, 0u);
+      if (c < nchunks) raw[i * V + j] = __ldg(reinterpret_cast<const uint4*>(src + (size_t)c * 8) + j);
+    }
+  }
+}
+
+template <typename T> __device__ __forceinline__ void row_unpack(const uint4 (&raw)[kRowRegs], int i, float (&v)[8]);
+template <> __device__ __forceinline__ void row_unpack<float>(const uint4 (&raw)[kRowRegs], int i, float (&v)[8]) {
+  const uint4 a = raw[2 * i], b = raw[2 * i + 1];
+  v[0] = __uint_as_float(a.x); v[1] = __uint_as_float(a.y); v[2] = __uint_as_float(a.z); v[3] = __uint_as_float(a.w);
+  v[4] = __uint_as_float(b.x); v[5] = __uint_as_float(b.y); v[6] = __uint_as_float(b.z); v[7] = __uint_as_float(b.w);
+}
+template <> __device__ __forceinline__ void row_unpack<__half>(const uint4 (&raw)[kRowRegs], int i, float (&v)[8]) {
+  const uint32_t w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[j]));
+    v[2 * j] = f.x; v[2 * j + 1] = f.y;
+  }
+}
+template <> __device__ __forceinline__ void row_unpack<__nv_bfloat16>(const uint4 (&raw)[kRowRegs], int i, float (&v)[8]) {
+  const uint32_t w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    v[2 * j] = __uint_as_float(w[j] << 16);
+    v[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+  }
+}
+
+struct RowStats { double mean, rstd; float xlo, xhi; };
+
+// Eq. 12 statistics of the segment held in raw[]: every lane returns the same values.
+template <typename T>
+__device__ __forceinline__ RowStats row_stats(const uint4 (&raw)[kRowRegs], int nchunks, int lane, float ln_eps,
+                                              double inv_kg) {
+  float s = 0.f, mn = INFINITY, mx = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < RowTraits<T>::kChunks; ++i) {
+    if (lane + 32 * i < nchunks) {
+      float v[8];
+      row_unpack<T>(raw, i, v);
+      s += ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { mn = fminf(mn, v[j]); mx = fmaxf(mx, v[j]); }
+    }
+  }
+  const double S = warp_sum((double)s);
+  RowStats st;
+  st.xlo = warp_min(mn); st.xhi = warp_max(mx);
+  if (ln_eps < 0.f) { st.mean = 0.0; st.rstd = 1.0; return st; }
+  st.mean = S * inv_kg;
+  const float mean_f = (float)st.mean;
+  float q = 0.f;
+#pragma unroll
+  for (int i = 0; i < RowTraits<T>::kChunks; ++i) {
+    if (lane + 32 * i < nchunks) {
+      float v[8];
+      row_unpack<T>(raw, i, v);
+      float p = 0.f;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { const float d = v[j] - mean_f; p = fmaf(d, d, p); }
+      q += p;
+    }
+  }
+  const double Q = warp_sum((double)q);
+  const double dm = st.mean - (double)mean_f;
+  double var = Q * inv_kg - dm * dm;                 // sum (x-mean)^2 = sum (x-mean_f)^2 - K dm^2
+  if (var < 0.0) var = 0.0;
+  st.rstd = rsqrt_newton(var + (double)ln_eps);
+  return st;
+}
+
+struct RowMap {            // Quant of Eq. 4-6 as one fp32 FMA, plus what the exact redo needs
+  double mean, rstd, eta, scale;
+  float A, B, tau;
+  int code_lo;
+};
+__device__ __forceinline__ RowMap row_map(int mode, double mean, double rstd, double gamma, double eta, float xabs) {
+  RowMap m;
+  m.mean = mean; m.rstd = rstd; m.eta = eta;
+  m.scale = gamma > 0.0 ? (double)kQb * rcp_newton(gamma) : 0.0;
+  m.A = (float)(rstd * m.scale);
+  m.B = (float)(-(mean * rstd + eta) * m.scale);
+  m.tau = 4e-7f * (fabsf(m.A) * xabs + fabsf(m.B) + 1.0f);
+  m.code_lo = (mode == BL_ABSMAX) ? -kCodeMax : 0;
+  return m;
+}
+// The rare element too close to a rounding tie for fp32: the equations in fp64, in their order.
+__device__ __noinline__ int row_code_exact(float x, double mean, double rstd, double eta, double scale) {
+  const double xh = ((double)x - mean) * rstd;
+  return (int)rint((xh - eta) * scale);
+}
+__device__ __forceinline__ uint2 row_codes8(const float (&v)[8], const RowMap& m) {
+  int code[8];
+  bool near_tie = false;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const float f = fmaf(v[j], m.A, m.B);
+    const float t = f + kRoundMagic;
+    const float r = t - kRoundMagic;
+    code[j] = __float_as_int(t) - __float_as_int(kRoundMagic);
+    near_tie |= fabsf(fabsf(f - r) - 0.5f) < m.tau;
+  }
+  if (near_tie) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) code[j] = row_code_exact(v[j], m.mean, m.rstd, m.eta, m.scale);
+  }
+  uint32_t w[2] = {0u, 0u};
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+    w[j >> 2] |= (uint32_t)(max(m.code_lo, min(kCodeMax, code[j])) & 0xFF) << (8 * (j & 3));
+  return make_uint2(w[0], w[1]);
+}
+
+template <typename T>
+__device__ __forceinline__ void row_store_codes(const uint4 (&raw)[kRowRegs], int nchunks, int lane, const RowMap& map,
+                                                int8_t* __restrict__ dst) {
+#pragma unroll
+  for (int i = 0; i < RowTraits<T>::kChunks; ++i) {
+    const int c = lane + 32 * i;
+    if (c < nchunks) {
+      float v[8];
+      row_unpack<T>(raw, i, v);
+      *reinterpret_cast<uint2*>(dst + (size_t)c * 8) = row_codes8(v, map);
+    }
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kRowWarps * 32, 2)
+rows_per_token(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg, int mode, float ln_eps,
+               double inv_kg, int8_t* __restrict__ x_q, float* __restrict__ gamma, float* __restrict__ eta) {
+  const int lane = threadIdx.x & 31;
+  const int64_t seg = (int64_t)blockIdx.x * kRowWarps + (threadIdx.x >> 5);
+  if (seg >= segments) return;                                   // whole warp
+  const int64_t base = (seg / G) * K + (seg % G) * (int64_t)Kg;
+  const int nchunks = Kg / 8;
+  uint4 raw[kRowRegs];
+  row_load<T>(x + base, nchunks, lane, raw);
+  const RowStats st = row_stats<T>(raw, nchunks, lane, ln_eps, inv_kg);
+  const double lo = ((double)st.xlo - st.mean) * st.rstd, hi = ((double)st.xhi - st.mean) * st.rstd;
+  double gam, et;
+  scope_gamma_eta(mode, lo, hi, gam, et);
+  const RowMap map = row_map(mode, st.mean, st.rstd, gam, et, fmaxf(fabsf(st.xlo), fabsf(st.xhi)));
+  if (lane == 0) {
+    gamma[seg] = (float)gam;
+    if (eta) eta[seg] = (float)et;
+  }
+  row_store_codes<T>(raw, nchunks, lane, map, x_q + base);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kRowWarps * 32, 2)
+rows_tensor_stats(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg, float ln_eps, double inv_kg,
+                  TensorScope* sc, SegRecord* __restrict__ recs) {
+  const int lane = threadIdx.x & 31;
+  const int64_t seg = (int64_t)blockIdx.x * kRowWarps + (threadIdx.x >> 5);
+  if (seg >= segments) return;
+  const int g = (int)(seg % G);
+  const int64_t base = (seg / G) * K + g * (int64_t)Kg;
+  const int nchunks = Kg / 8;
+  uint4 raw[kRowRegs];
+  row_load<T>(x + base, nchunks, lane, raw);
+  const RowStats st = row_stats<T>(raw, nchunks, lane, ln_eps, inv_kg);
+  if (lane == 0) {
+    recs[seg] = SegRecord{st.mean, st.rstd, fmaxf(fabsf(st.xlo), fabsf(st.xhi)), 0.f};
+    atomicMin(&sc->enc_min[g], enc_ordered64(((double)st.xlo - st.mean) * st.rstd));
+    atomicMax(&sc->enc_max[g], enc_ordered64(((double)st.xhi - st.mean) * st.rstd));
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kRowWarps * 32, 2)
+rows_tensor_codes(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg, int mode,
+                  const TensorScope* __restrict__ sc, const SegRecord* __restrict__ recs,
+                  int8_t* __restrict__ x_q, float* __restrict__ gamma, float* __restrict__ eta) {
+  const int lane = threadIdx.x & 31;
+  const int64_t seg = (int64_t)blockIdx.x * kRowWarps + (threadIdx.x >> 5);
+  if (seg >= segments) return;
+  const int g = (int)(seg % G);
+  const int64_t base = (seg / G) * K + g * (int64_t)Kg;
+  const int nchunks = Kg / 8;
+  uint4 raw[kRowRegs];
+  row_load<T>(x + base, nchunks, lane, raw);                      // in flight during the scalar work below
+  const SegRecord rec = recs[seg];
+  const double lo = dec_ordered64(sc->enc_min[g]), hi = dec_ordered64(sc->enc_max[g]);
+  double gam, et;
+  scope_gamma_eta(mode, lo, hi, gam, et);
+  const RowMap map = row_map(mode, rec.mean, rec.rstd, gam, et, rec.xabs);
+  if (seg < G && lane == 0) {                                      // token 0 reports the scope's gamma / eta
+    gamma[g] = (float)gam;
+    if (eta) eta[g] = (float)et;
+  }
+  row_store_codes<T>(raw, nchunks, lane, map, x_q + base);
+}
+
 template <typename T>
 cudaError_t run(const QuantArgs& a, cudaStream_t s) {
   const T* x = reinterpret_cast<const T*>(a.x);
@@ -127,6 +368,23 @@ cudaError_t run(const QuantArgs& a, cudaStream_t s) {
   const size_t smem = (size_t)Kg * sizeof(float);
   const unsigned grid = (unsigned)(a.M * a.G);
   cudaError_t e;
+  if (Kg <= RowTraits<T>::kMaxKg) {                              // a segment fits a warp's registers
+    const int64_t segments = a.M * a.G;
+    const unsigned rgrid = (unsigned)((segments + kRowWarps - 1) / kRowWarps);
+    const double inv_kg = 1.0 / (double)Kg;
+    if (a.gran == BL_PER_TOKEN) {
+      rows_per_token<T><<<rgrid, kRowWarps * 32, 0, s>>>(x, segments, a.K, a.G, (int)Kg, (int)a.mode, a.ln_eps,
+                                                         inv_kg, a.x_q, a.gamma, a.eta);
+      return cudaGetLastError();
+    }
+    TensorScope* sc = reinterpret_cast<TensorScope*>(a.ws);
+    SegRecord* recs = reinterpret_cast<SegRecord*>(reinterpret_cast<char*>(a.ws) + sizeof(TensorScope));
+    init_scope<<<1, BL_MAX_GROUPS, 0, s>>>(sc);
+    rows_tensor_stats<T><<<rgrid, kRowWarps * 32, 0, s>>>(x, segments, a.K, a.G, (int)Kg, a.ln_eps, inv_kg, sc, recs);
+    rows_tensor_codes<T><<<rgrid, kRowWarps * 32, 0, s>>>(x, segments, a.K, a.G, (int)Kg, (int)a.mode, sc, recs,
+                                                          a.x_q, a.gamma, a.eta);
+    return cudaGetLastError();
+  }
   if (a.gran == BL_PER_TOKEN) {
     if (smem > 48 * 1024) {
       e = cudaFuncSetAttribute(quant_per_token<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
