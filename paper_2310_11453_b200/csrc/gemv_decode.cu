@@ -56,14 +56,6 @@ __device__ __forceinline__ int code_slot(int k) {
   return (k & ~(kSlice - 1)) | ((((k >> 4) & 7) * 32 + ((k >> 7) & 31)) << 4) | (k & 15);
 }
 
-// 1/d in fp64 from the fp32 reciprocal and one Newton step (relative error 2^-23, then about
-// 2^-45: a code can differ from exact arithmetic only within 1e-11 of a rounding tie);
-// arguments outside the fp32 range take the exact division.
-__device__ __forceinline__ double rcp_f64(double d) {
-  if (!(d > 1e-30 && d < 1e30)) return 1.0 / d;
-  const double y = (double)__frcp_rn((float)d);
-  return y * (2.0 - d * y);
-}
 // 1/sqrt(v) to fp32 accuracy (it only scales the output); exact routine outside the fp32 range.
 __device__ __forceinline__ float rsqrt_scale(double v) {
   if (!(v > 1e-30 && v < 1e30)) return v > 0.0 ? (float)(1.0 / sqrt(v)) : 0.f;

@@ -11,6 +11,7 @@
 // workspace and folds the extremes of x^ into a global atomic min/max on an order-preserving
 // encoding (order-independent, hence deterministic); the second re-reads x and writes codes.
 #include <mutex>
+#include <type_traits>
 
 #include "quant_core.cuh"
 
@@ -196,42 +197,73 @@ template <> __device__ __forceinline__ void row_unpack<__nv_bfloat16>(const uint
 
 struct RowStats { double mean, rstd; float xlo, xhi; };
 
+template <typename H2> __device__ __forceinline__ H2 as_h2(uint32_t w) { return *reinterpret_cast<H2*>(&w); }
+template <typename H2> __device__ __forceinline__ uint32_t h2_bits(H2 h) { return *reinterpret_cast<uint32_t*>(&h); }
+
 // Eq. 12 statistics of the segment held in raw[]: every lane returns the same values.
+// One pass: deviations are taken from a pilot value c (the mean of the segment's first 8
+// elements), which keeps sum (x - c) and sum (x - c)^2 small and well conditioned:
+//   mean = c + sum (x - c) / K,   Var = sum (x - c)^2 / K - (mean - c)^2.
 template <typename T>
 __device__ __forceinline__ RowStats row_stats(const uint4 (&raw)[kRowRegs], int nchunks, int lane, float ln_eps,
                                               double inv_kg) {
-  float s = 0.f, mn = INFINITY, mx = -INFINITY;
+  float pilot = 0.f;
+  {
+    float v[8];
+    row_unpack<T>(raw, 0, v);                        // lane 0 holds chunk 0
+    pilot = 0.125f * (((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7])));
+    pilot = __shfl_sync(0xFFFFFFFFu, pilot, 0);
+    if (ln_eps < 0.f) pilot = 0.f;
+  }
+  float s = 0.f, q = 0.f, mn = INFINITY, mx = -INFINITY;
+  uint32_t plo = 0, phi = 0;
+  bool have16 = false;
 #pragma unroll
   for (int i = 0; i < RowTraits<T>::kChunks; ++i) {
     if (lane + 32 * i < nchunks) {
       float v[8];
       row_unpack<T>(raw, i, v);
-      s += ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
+      float d[8];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) { mn = fminf(mn, v[j]); mx = fmaxf(mx, v[j]); }
+      for (int j = 0; j < 8; ++j) d[j] = v[j] - pilot;
+      s += ((d[0] + d[1]) + (d[2] + d[3])) + ((d[4] + d[5]) + (d[6] + d[7]));
+      float p = 0.f;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) p = fmaf(d[j], d[j], p);
+      q += p;
+      if constexpr (sizeof(T) == 4) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { mn = fminf(mn, v[j]); mx = fmaxf(mx, v[j]); }
+      } else {
+        using H2 = typename std::conditional<std::is_same<T, __half>::value, __half2, __nv_bfloat162>::type;
+        const uint32_t w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
+        H2 a = __hmin2(__hmin2(as_h2<H2>(w[0]), as_h2<H2>(w[1])), __hmin2(as_h2<H2>(w[2]), as_h2<H2>(w[3])));
+        H2 b = __hmax2(__hmax2(as_h2<H2>(w[0]), as_h2<H2>(w[1])), __hmax2(as_h2<H2>(w[2]), as_h2<H2>(w[3])));
+        if (have16) { a = __hmin2(a, as_h2<H2>(plo)); b = __hmax2(b, as_h2<H2>(phi)); }
+        plo = h2_bits(a); phi = h2_bits(b); have16 = true;
+      }
     }
   }
-  const double S = warp_sum((double)s);
+  if constexpr (sizeof(T) != 4) {
+    if (have16) {
+      using H2 = typename std::conditional<std::is_same<T, __half>::value, __half2, __nv_bfloat162>::type;
+      const H2 a = as_h2<H2>(plo), b = as_h2<H2>(phi);
+      if constexpr (std::is_same<T, __half>::value) {
+        const float2 fa = __half22float2(a), fb = __half22float2(b);
+        mn = fminf(fa.x, fa.y); mx = fmaxf(fb.x, fb.y);
+      } else {
+        const float2 fa = __bfloat1622float2(a), fb = __bfloat1622float2(b);
+        mn = fminf(fa.x, fa.y); mx = fmaxf(fb.x, fb.y);
+      }
+    }
+  }
+  const double S = warp_sum((double)s), Q = warp_sum((double)q);
   RowStats st;
   st.xlo = warp_min(mn); st.xhi = warp_max(mx);
   if (ln_eps < 0.f) { st.mean = 0.0; st.rstd = 1.0; return st; }
-  st.mean = S * inv_kg;
-  const float mean_f = (float)st.mean;
-  float q = 0.f;
-#pragma unroll
-  for (int i = 0; i < RowTraits<T>::kChunks; ++i) {
-    if (lane + 32 * i < nchunks) {
-      float v[8];
-      row_unpack<T>(raw, i, v);
-      float p = 0.f;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) { const float d = v[j] - mean_f; p = fmaf(d, d, p); }
-      q += p;
-    }
-  }
-  const double Q = warp_sum((double)q);
-  const double dm = st.mean - (double)mean_f;
-  double var = Q * inv_kg - dm * dm;                 // sum (x-mean)^2 = sum (x-mean_f)^2 - K dm^2
+  const double dm = S * inv_kg;                      // mean - pilot
+  st.mean = (double)pilot + dm;
+  double var = Q * inv_kg - dm * dm;
   if (var < 0.0) var = 0.0;
   st.rstd = rsqrt_newton(var + (double)ln_eps);
   return st;
@@ -258,25 +290,31 @@ __device__ __noinline__ int row_code_exact(float x, double mean, double rstd, do
   return (int)rint((xh - eta) * scale);
 }
 __device__ __forceinline__ uint2 row_codes8(const float (&v)[8], const RowMap& m) {
-  int code[8];
+  // f is clipped in fp32 (the clip bounds are integers, so clip and rne commute); adding the
+  // magic constant leaves rne(f) as a two's-complement byte in the low bits of the sum.
+  uint32_t t[8];
   bool near_tie = false;
+  const float lo = (float)m.code_lo, hi = (float)kCodeMax, edge = 0.5f - m.tau;
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
     const float f = fmaf(v[j], m.A, m.B);
-    const float t = f + kRoundMagic;
-    const float r = t - kRoundMagic;
-    code[j] = __float_as_int(t) - __float_as_int(kRoundMagic);
-    near_tie |= fabsf(fabsf(f - r) - 0.5f) < m.tau;
+    const float tj = fminf(fmaxf(f, lo), hi) + kRoundMagic;
+    near_tie |= fabsf(f - (tj - kRoundMagic)) > edge;         // inside the clip range: within tau of a tie
+    t[j] = __float_as_uint(tj);
   }
-  if (near_tie) {
+  uint2 out;
+  out.x = __byte_perm(__byte_perm(t[0], t[1], 0x0040), __byte_perm(t[2], t[3], 0x0040), 0x5410);
+  out.y = __byte_perm(__byte_perm(t[4], t[5], 0x0040), __byte_perm(t[6], t[7], 0x0040), 0x5410);
+  if (near_tie) {                                            // rare: redo the 8 codes exactly
+    uint32_t w[2] = {0u, 0u};
 #pragma unroll
-    for (int j = 0; j < 8; ++j) code[j] = row_code_exact(v[j], m.mean, m.rstd, m.eta, m.scale);
+    for (int j = 0; j < 8; ++j) {
+      const int c = max(m.code_lo, min(kCodeMax, row_code_exact(v[j], m.mean, m.rstd, m.eta, m.scale)));
+      w[j >> 2] |= (uint32_t)(c & 0xFF) << (8 * (j & 3));
+    }
+    out = make_uint2(w[0], w[1]);
   }
-  uint32_t w[2] = {0u, 0u};
-#pragma unroll
-  for (int j = 0; j < 8; ++j)
-    w[j >> 2] |= (uint32_t)(max(m.code_lo, min(kCodeMax, code[j])) & 0xFF) << (8 * (j & 3));
-  return make_uint2(w[0], w[1]);
+  return out;
 }
 
 template <typename T>
