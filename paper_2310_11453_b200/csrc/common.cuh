@@ -133,6 +133,7 @@ struct GemmArgs {
 };
 cudaError_t launch_gemm_simple(const GemmArgs& a, cudaStream_t s);
 cudaError_t launch_gemm_tc(const GemmArgs& a, cudaStream_t s);
+cudaError_t launch_gemm_tc2(const GemmArgs& a, cudaStream_t s);   // two SMs per tile
 bool gemm_tc_supported(int64_t M, int64_t K, int64_t N, int G);
 size_t gemm_tc_scratch_bytes(int64_t M, int64_t N, int G);   // host-only, no device query
 
