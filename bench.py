@@ -246,8 +246,8 @@ def run_b200(args):
         "clocks": None,
         "e2e": e2e,
         "gpu_launches": 4 * K_steps,
-        "kernels_per_step": ["init_scope", "rows_tensor_stats", "rows_tensor_codes", "gemm_tc_kernel"],
-        "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": gemm_tops, "peak": tensor_peak,
+        "kernels_per_step": ["init_scope", "rows_tensor_stats", "rows_tensor_codes", "gemm_tc2_kernel"],
+        "roofline": {"bound": "tensor", "kernel": "gemm_tc2_kernel", "achieved": gemm_tops, "peak": tensor_peak,
                      "unit": "TFLOP/s", "frac": gemm_tops / tensor_peak, "traffic": None,
                      "op_kind": "int8 (s8 x s8 -> s32), 2 ops per multiply-accumulate",
                      "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} x {INT8_TO_BF16} "

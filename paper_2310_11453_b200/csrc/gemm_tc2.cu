@@ -18,11 +18,12 @@
 //   warps 4-7   epilogue
 //   warps 8-15  weight expanders: two groups of 4 warps on alternate stages, thread u of a group
 //               owns row u of this CTA's 128-row half of the B tile
-// Barriers.  In every CTA: full_a (own TMA bytes), empty (stage consumed; the issuer commits to
-// both CTAs' copies), tmem_full (accumulator complete; committed to both).  Only in rank 0, with
-// arrivals from both CTAs: peer_a (rank 1's codes landed), full_b (8 expander warps), tmem_empty
-// (8 epilogue warps).  Remote arrivals are mbarrier.arrive.release.cluster on the mapa address;
-// the waits that see them acquire at cluster scope.
+// Barriers.  In every CTA: empty (stage consumed; the issuer commits to both CTAs' copies) and
+// tmem_full (accumulator complete; committed to both).  full: in rank 0 one barrier per stage
+// collects its own TMA bytes, rank 1's "codes landed" and the 8 expander warps of the pair, so the
+// issuer - whose serial per-stage work bounds the whole kernel - waits once per stage; in rank 1
+// it tracks that CTA's TMA only.  tmem_empty (rank 0) takes the 8 epilogue warps of the pair.
+// Remote arrivals are mbarrier.arrive on the mapa address of rank 0's barrier.
 //
 // Every wait is bounded; a limit that runs out raises the CTA's abort flag, records
 // BL_ERR_TIMEOUT and lets every role fall through to the common exit (cluster barrier, tensor
@@ -52,8 +53,8 @@ constexpr int kMaxCtas = 160;
 constexpr size_t kScratchPerCta = (size_t)kBM * kBN * sizeof(float);
 
 struct SharedCtl {
-  unsigned long long full_a[kStages], empty[kStages];
-  unsigned long long peer_a[kStages], full_b[kStages];          // used in rank 0 only
+  unsigned long long full[kStages];      // rank 0: everything a stage needs (see below); rank 1: own TMA bytes
+  unsigned long long empty[kStages];
   unsigned long long tmem_full[2], tmem_empty[2];               // tmem_empty used in rank 0 only
   uint32_t tmem_base;
   int abort_flag;
@@ -77,30 +78,13 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t ra
   return r;
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\n"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait with cluster-scope acquire (sees arrivals and commits made by the partner CTA).
+// Waits on barriers that the partner CTA (or a tcgen05.commit of the pair) arrives on use the same
+// bounded CTA-scope wait as local ones: what crosses CTAs here is only the barrier count itself;
+// the data behind it is read by the tensor core (async proxy), not by this CTA's threads.
 __device__ __forceinline__ bool mbar_wait2(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try_wait_cluster(bar, parity)) return true;
-  const unsigned long long t0 = global_ns();
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
-    if (mbar_try_wait_cluster(bar, parity)) return true;
-    if ((it & 255u) == 255u) {
-      if (*abort_flag) return false;
-      if (global_ns() - t0 > kWaitNs) break;
-    }
-  }
-  *abort_flag = 1;
-  return false;
+  return mbar_wait(bar, parity, abort_flag);
 }
 __device__ __forceinline__ void mma_i8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                             uint32_t accumulate) {
@@ -150,10 +134,11 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
-      mbar_init(smem_u32(&ctl->full_a[s]), 1);
+      // rank 0's full barrier collects, per stage: its own TMA (1 arrival + the bytes), rank 1's
+      // "codes landed" (1) and the expander warps of both CTAs (2 x 4), so the MMA issuer makes
+      // one wait per stage.  Rank 1's copy only tracks its own TMA.
+      mbar_init(smem_u32(&ctl->full[s]), leader ? 2 + 2 * (kHalfN / 32) : 1);
       mbar_init(smem_u32(&ctl->empty[s]), 1);
-      mbar_init(smem_u32(&ctl->peer_a[s]), 1);
-      mbar_init(smem_u32(&ctl->full_b[s]), 2 * (kHalfN / 32));
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&ctl->tmem_full[b]), 1);
@@ -183,7 +168,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
         const int m0 = (int)(it.m_tile() * kPairM + rank * kBM);
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!mbar_wait2(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
-          const uint32_t bar = smem_u32(&ctl->full_a[stage]);
+          const uint32_t bar = smem_u32(&ctl->full[stage]);
           mbar_arrive_expect_tx(bar, (uint32_t)tx_bytes);
           tma_load_2d(smem_u32(smem + (size_t)stage * kStageBytes), &map_x, kb * kBK, m0, bar);
           ++issued;
@@ -195,7 +180,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
       for (uint32_t i = 0; i < pending; ++i) {
         if (stage == 0) { stage = kStages; phase ^= 1u; }
         --stage;
-        (void)mbar_wait(smem_u32(&ctl->full_a[stage]), phase, abort_flag);
+        (void)mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag);
       }
     }
   } else if (warp == 1 && !leader) {
@@ -205,8 +190,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
       bool ok = true;
       for (PairIter it(tiles, m_tiles); ok && it.valid(); it.next()) {
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!mbar_wait(smem_u32(&ctl->full_a[stage]), phase, abort_flag)) { ok = false; break; }
-          mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->peer_a[stage]), 0));
+          if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
+          mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->full[stage]), 0));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -217,6 +202,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
       int stage = 0; uint32_t phase = 0;
       uint32_t pass = 0;
       bool ok = true;
+      const uint32_t empty0 = map_to_rank(smem_u32(&ctl->empty[0]), 0), empty1 = map_to_rank(smem_u32(&ctl->empty[0]), 1);
       for (PairIter it(tiles, m_tiles); ok && it.valid(); it.next()) {
         for (int g = 0; ok && g < a.G; ++g, ++pass) {
           const uint32_t buf = pass & 1u, acc_phase = (pass >> 1) & 1u;
@@ -224,9 +210,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + buf * (uint32_t)kBN;
           for (int kb = 0; kb < kb_per_group; ++kb) {
-            if (!mbar_wait(smem_u32(&ctl->full_a[stage]), phase, abort_flag) ||
-                !mbar_wait2(smem_u32(&ctl->peer_a[stage]), phase, abort_flag) ||
-                !mbar_wait2(smem_u32(&ctl->full_b[stage]), phase, abort_flag)) { ok = false; break; }
+            if (!mbar_wait2(smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
             tc_fence_after();
             const uint32_t a_addr = smem_u32(smem + (size_t)stage * kStageBytes);
             const uint64_t adesc = smem_desc_sw128(a_addr);
@@ -235,9 +219,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
             for (int j = 0; j < kBK / 32; ++j)
               mma_i8_pair(d_tmem, adesc + (uint64_t)(2 * j), bdesc + (uint64_t)(2 * j), kIdesc,
                           (kb > 0 || j > 0) ? 1u : 0u);
-            const uint32_t e = smem_u32(&ctl->empty[stage]);
-            mma_commit_pair(map_to_rank(e, 0));
-            mma_commit_pair(map_to_rank(e, 1));
+            mma_commit_pair(empty0 + 8u * (uint32_t)stage);
+            mma_commit_pair(empty1 + 8u * (uint32_t)stage);
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
           if (ok) {
@@ -254,6 +237,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
     const int u = (threadIdx.x - kExpandWarp0 * 32) & (kHalfN - 1);  // row of this CTA's half, 0..127
     const uint32_t row_base = smem_u32(smem) + (uint32_t)kABytes + (uint32_t)u * 128u + ((uint32_t)(u & 7) << 4);
     int stage = eg; uint32_t phase = 0;
+    const uint32_t full0 = map_to_rank(smem_u32(&ctl->full[0]), 0);
     PairIter pf_it(tiles, m_tiles);
     int pf_kb = eg;
     const uint8_t* pf_src = nullptr;                                 // row u of the tile's first k-block
@@ -301,7 +285,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
       }
       fence_proxy_async_smem();
       __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->full_b[stage]), 0));
+      if (lane == 0) mbar_arrive_cluster(full0 + 8u * (uint32_t)stage);
       stage += 2;
       if (stage >= kStages) { stage -= kStages; phase ^= 1u; }
     }
@@ -425,6 +409,24 @@ cudaError_t launch(const GemmArgs& a, cudaStream_t s) {
   const int64_t tiles = ((a.M + kPairM - 1) / kPairM) * ((a.N + kBN - 1) / kBN);
   if (tiles >= (int64_t)1 << 31) return cudaErrorInvalidValue;
   int64_t clusters = (sms < kMaxCtas ? sms : kMaxCtas) / 2;
+  {
+    // persistent grid: no more clusters than can be resident at once
+    static int resident[2][3] = {};
+    if (resident[kMode][ti] == 0) {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3((unsigned)(2 * clusters));
+      cfg.blockDim = dim3(kThreads);
+      cfg.dynamicSmemBytes = kSmemBytes;
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+      cfg.attrs = at; cfg.numAttrs = 1;
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n < 1) { (void)cudaGetLastError(); n = (int)clusters; }
+      resident[kMode][ti] = n;
+    }
+    if (resident[kMode][ti] < clusters) clusters = resident[kMode][ti];
+  }
   if (tiles < clusters) clusters = tiles;
   kern<<<(unsigned)(2 * clusters), kThreads, kSmemBytes, s>>>(map, a, (int)(box_m * kBK));
   return cudaGetLastError();
