@@ -10,14 +10,14 @@
 // halves.  Compared with one SM per tile this halves, per SM, the expansion arithmetic, the
 // expansion stores and the tensor core's reads of B.
 //
-// Roles per CTA (16 warps):
+// Roles per CTA:
 //   warp 0      TMA producer for this CTA's codes tile
 //   warp 1      rank 0: MMA issuer for the pair (one thread); rank 1: forwards "my codes tile has
 //               landed" to rank 0's barrier
 //   warp 2      tensor-memory allocation (both CTAs, cta_group::2)
 //   warps 4-7   epilogue
-//   warps 8-15  weight expanders: two groups of 4 warps on alternate stages, thread u of a group
-//               owns row u of this CTA's 128-row half of the B tile
+//   warps 8-..  weight expanders: groups of 4 warps, group e on stages e, e + groups, ...; thread u
+//               of a group owns row u of this CTA's 128-row half of the B tile
 // Barriers.  In every CTA: empty (stage consumed; the issuer commits to both CTAs' copies) and
 // tmem_full (accumulator complete; committed to both).  full: in rank 0 one barrier per stage
 // collects its own TMA bytes, rank 1's "codes landed" and the 8 expander warps of the pair, so the
@@ -42,8 +42,13 @@ constexpr int kBN = 256;                 // output features per tile (MMA N)
 constexpr int kHalfN = 128;              // weight rows expanded per CTA
 constexpr int kBK = 128;                 // weights per stage (one 128-byte swizzle atom)
 constexpr int kStages = 6;
-constexpr int kThreads = 512;
+#ifndef BL_GEMM_EXPAND_GROUPS
+#define BL_GEMM_EXPAND_GROUPS 2
+#endif
+constexpr int kGroups = BL_GEMM_EXPAND_GROUPS;   // expander groups of 4 warps; group e takes stages e, e + kGroups, ..
+static_assert(kStages % kGroups == 0, "every stage must belong to one group");
 constexpr int kExpandWarp0 = 8;
+constexpr int kThreads = (kExpandWarp0 + 4 * kGroups) * 32;
 constexpr int kEpiWarp0 = 4;
 constexpr int kABytes = kBM * kBK;       // 16 KB
 constexpr int kBBytes = kHalfN * kBK;    // 16 KB
@@ -233,7 +238,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
     }
   } else if (warp >= kExpandWarp0) {
     // ---------------------------------------------------------------- weight expanders (own half of B)
-    const int eg = (warp - kExpandWarp0) >> 2;                       // group 0 or 1
+    const int eg = (warp - kExpandWarp0) >> 2;                       // group number
     const int u = (threadIdx.x - kExpandWarp0 * 32) & (kHalfN - 1);  // row of this CTA's half, 0..127
     const uint32_t row_base = smem_u32(smem) + (uint32_t)kABytes + (uint32_t)u * 128u + ((uint32_t)(u & 7) << 4);
     int stage = eg; uint32_t phase = 0;
@@ -254,7 +259,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
       if (pf_it.valid()) {
         if (pf_src) v = __ldg(reinterpret_cast<const uint4*>(pf_src + (size_t)pf_kb * 2048));
-        pf_kb += 2;
+        pf_kb += kGroups;
         if (pf_kb >= k_blocks) seek();
       }
       return v;
@@ -263,7 +268,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
     const uint32_t nclusters = gridDim.x >> 1, cid = blockIdx.x >> 1;
     const uint32_t my_tiles = (tiles > cid) ? (tiles - cid + nclusters - 1) / nclusters : 0u;
     const uint64_t flat = (uint64_t)my_tiles * (uint64_t)k_blocks;
-    const uint64_t owned = flat > (uint64_t)eg ? (flat - eg + 1) / 2 : 0;
+    const uint64_t owned = flat > (uint64_t)eg ? (flat - eg + kGroups - 1) / kGroups : 0;
     for (uint64_t i = 0; i < owned; ++i) {
       const uint4 cur = b0;
       b0 = b1;
@@ -286,7 +291,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(full0 + 8u * (uint32_t)stage);
-      stage += 2;
+      stage += kGroups;
       if (stage >= kStages) { stage -= kStages; phase ^= 1u; }
     }
   } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + 4) {
