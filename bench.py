@@ -264,6 +264,8 @@ def run_b200(args):
             line["decode"] = bench_decode(B, synth, dev, peaks)
         if "pack" in parts:
             line["pack"] = bench_pack(B, synth, dev, peaks)
+        if "grouped" in parts:
+            line["grouped"] = bench_grouped(B, synth, dev, peaks)
         if "cpu" in parts:
             line["cpu_baseline"] = cpu_baseline_prefill(xs_host[0], W.cpu())
     line["clocks"] = clocks.summary()
@@ -378,6 +380,53 @@ def bench_pack(B, synth, dev, peaks):
                          "peak_source": peaks["source"] + " copy"}}
 
 
+def bench_grouped(B, synth, dev, peaks):
+    """Config 5: 30B-shaped FFN down-projection with group quantization, G = 8 along K.  Binarize+pack,
+    LN+quant (eta form, per-group scalars over all tokens) and the full forward, each timed alone."""
+    M, K, N, G = 4096, 28672, 7168, 8
+    W = synth.make_w(N, K, torch.float32, seed=4).to(dev)
+    x = synth.make_x(M, K, torch.bfloat16, seed=4, outliers=False, relu=True).to(dev)
+    w = B.binarize_pack(W, G=G, layout=B.PREFILL)
+    ws_p = torch.empty(B.workspace_bytes(B.OP_BINARIZE_PACK, 1, N, K, G), dtype=torch.uint8, device=dev)
+    ws_q = torch.empty(B.workspace_bytes(B.OP_QUANT_ACT, M, 1, K, G), dtype=torch.uint8, device=dev)
+    ws_f = torch.empty(B.workspace_bytes(B.OP_FORWARD, M, N, K, G), dtype=torch.uint8, device=dev)
+    q = dict(x_q=torch.empty((M, K), dtype=torch.int8, device=dev),
+             gamma=torch.empty(G, dtype=torch.float32, device=dev), eta=torch.empty(G, dtype=torch.float32, device=dev))
+    y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+
+    def timed(fn, reps):
+        for _ in range(2):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    t_pack = timed(lambda: B.binarize_pack(W, G=G, layout=B.PREFILL, out=w, ws=ws_p), 5)
+    t_quant = timed(lambda: B.quant_act(x, G=G, mode=B.ETA, gran=B.PER_TENSOR, out=q, ws=ws_q), 5)
+    t_gemm = timed(lambda: B.matmul_dequant(q["x_q"], q["gamma"], w["W_packed"], w["beta"], N, G=G,
+                                            gran=B.PER_TENSOR, layout=B.PREFILL, y=y, ws=ws_f), 5)
+    t_fwd = timed(lambda: B.forward(x, w["W_packed"], w["beta"], N, G=G, mode=B.ETA, gran=B.PER_TENSOR,
+                                    layout=B.PREFILL, y=y, ws=ws_f), 5)
+    assert B.ws_status(ws_f) == B.OK
+    pack_bytes = 2.0 * N * K * 4 + N * K / 8
+    quant_bytes = 2.0 * M * K * 2 + M * K
+    ops = 2.0 * M * N * K
+    tensor_peak = INT8_TO_BF16 * peaks["bf16_tflops"]
+    return {"workload": "30B-shaped FFN down-projection, G = 8 groups along K: W fp32 [7168,28672], x bf16 "
+                        "[4096,28672] = ReLU(N(0,1)), eta form, per-group alpha/beta/gamma/eta, y bf16; working "
+                        "sets exceed L2",
+            "pack_ms": t_pack, "pack_gbs": pack_bytes / t_pack / 1e6, "pack_frac": pack_bytes / t_pack / 1e6 / peaks["hbm_gbs"],
+            "quant_ms": t_quant, "quant_gbs": quant_bytes / t_quant / 1e6,
+            "quant_frac": quant_bytes / t_quant / 1e6 / peaks["hbm_gbs"],
+            "gemm_ms": t_gemm, "gemm_tops": ops / t_gemm / 1e9, "gemm_frac": ops / t_gemm / 1e9 / tensor_peak,
+            "forward_ms": t_fwd, "forward_tops": ops / t_fwd / 1e9}
+
+
 # --------------------------------------------------------------------------- the CPU oracle, timed
 
 def oracle_prefill_sample(x_host, W_host, tokens, reps=1):
@@ -462,8 +511,8 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
-    ap.add_argument("--parts", default="decode,pack,cpu",
-                    help="extra measurements beside the prefill step (comma list of decode, pack, cpu; "
+    ap.add_argument("--parts", default="decode,pack,grouped,cpu",
+                    help="extra measurements beside the prefill step (comma list of decode, pack, grouped, cpu; "
                          "'none' for the prefill step alone, e.g. under a profiler)")
     args = ap.parse_args()
     if args.impl == "reference":
