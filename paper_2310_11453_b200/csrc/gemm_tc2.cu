@@ -16,12 +16,14 @@
 //               landed" to rank 0's barrier
 //   warp 2      tensor-memory allocation (both CTAs, cta_group::2)
 //   warps 4-7   epilogue
-//   warps 8-..  weight expanders: groups of 4 warps, group e on stages e, e + groups, ...; thread u
-//               of a group owns row u of this CTA's 128-row half of the B tile
+//   warps 8-15  weight expanders: two groups of 4 warps, group e fills k-block e of every ring slot;
+//               thread u of a group owns row u of this CTA's 128-row half of the B tile
+// A ring slot holds two k-blocks (256 weights): the MMA issuer, whose serial work per barrier round
+// trip bounds the kernel, waits and commits once per slot and issues 8 MMAs in between.
 // Barriers.  In every CTA: empty (stage consumed; the issuer commits to both CTAs' copies) and
-// tmem_full (accumulator complete; committed to both).  full: in rank 0 one barrier per stage
+// tmem_full (accumulator complete; committed to both).  full: in rank 0 one barrier per slot
 // collects its own TMA bytes, rank 1's "codes landed" and the 8 expander warps of the pair, so the
-// issuer - whose serial per-stage work bounds the whole kernel - waits once per stage; in rank 1
+// issuer waits once per slot; in rank 1
 // it tracks that CTA's TMA only.  tmem_empty (rank 0) takes the 8 epilogue warps of the pair.
 // Remote arrivals are mbarrier.arrive on the mapa address of rank 0's barrier.
 //
@@ -40,31 +42,29 @@ constexpr int kBM = 128;                 // tokens per CTA (tensor-memory lanes)
 constexpr int kPairM = 256;              // tokens per tile
 constexpr int kBN = 256;                 // output features per tile (MMA N)
 constexpr int kHalfN = 128;              // weight rows expanded per CTA
-constexpr int kBK = 128;                 // weights per stage (one 128-byte swizzle atom)
-constexpr int kStages = 6;
-#ifndef BL_GEMM_EXPAND_GROUPS
-#define BL_GEMM_EXPAND_GROUPS 2
-#endif
-constexpr int kGroups = BL_GEMM_EXPAND_GROUPS;   // expander groups of 4 warps; group e takes stages e, e + kGroups, ..
-static_assert(kStages % kGroups == 0, "every stage must belong to one group");
+constexpr int kBK = 128;                 // weights per k-block (one 128-byte swizzle atom)
+constexpr int kSub = 2;                  // k-blocks per ring slot: one barrier round trip per 256 weights
+constexpr int kSlots = 3;                // ring slots of kSub x (codes tile + weights half-tile)
+constexpr int kGroups = kSub;            // expander groups of 4 warps; group e fills k-block e of every slot
 constexpr int kExpandWarp0 = 8;
 constexpr int kThreads = (kExpandWarp0 + 4 * kGroups) * 32;
 constexpr int kEpiWarp0 = 4;
 constexpr int kABytes = kBM * kBK;       // 16 KB
 constexpr int kBBytes = kHalfN * kBK;    // 16 KB
-constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kStageBytes = kABytes + kBBytes;   // one k-block
+constexpr int kSlotBytes = kSub * kStageBytes;
 constexpr int kTmemCols = 512;
 constexpr int kMaxCtas = 160;
 constexpr size_t kScratchPerCta = (size_t)kBM * kBN * sizeof(float);
 
 struct SharedCtl {
-  unsigned long long full[kStages];      // rank 0: everything a stage needs (see below); rank 1: own TMA bytes
-  unsigned long long empty[kStages];
+  unsigned long long full[kSlots];       // rank 0: everything a slot needs (see below); rank 1: own TMA bytes
+  unsigned long long empty[kSlots];
   unsigned long long tmem_full[2], tmem_empty[2];               // tmem_empty used in rank 0 only
   uint32_t tmem_base;
   int abort_flag;
 };
-constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 + sizeof(SharedCtl) + 64;
+constexpr size_t kSmemBytes = (size_t)kSlots * kSlotBytes + 1024 + sizeof(SharedCtl) + 64;
 static_assert(kSmemBytes <= 232448, "exceeds the shared memory of one CTA");
 
 // kind::i8 instruction descriptor: s32 accumulate, s8 x s8, both operands K-major, 256 x 256.
@@ -117,6 +117,21 @@ struct PairIter {            // tiles of this cluster, in the order every role o
   __device__ uint32_t n_tile() const { return t / m_tiles; }
 };
 
+// One ring slot's worth of work: up to kSub consecutive k-blocks of one (tile, group).  Every role
+// of both CTAs walks the same sequence of steps.
+struct StepIter {
+  PairIter it;
+  int g, t, G, spg, kbg;                      // group, step in group; groups, steps per group, k-blocks per group
+  __device__ StepIter(uint32_t tiles, uint32_t m_tiles, int G_, int kbg_)
+      : it(tiles, m_tiles), g(0), t(0), G(G_), spg((kbg_ + kSub - 1) / kSub), kbg(kbg_) {}
+  __device__ bool valid() const { return it.valid(); }
+  __device__ void next() { if (++t == spg) { t = 0; if (++g == G) { g = 0; it.next(); } } }
+  __device__ int nblk() const { const int r = kbg - t * kSub; return r < kSub ? r : kSub; }
+  __device__ int kb0() const { return g * kbg + t * kSub; }   // first k-block of the step
+  __device__ bool first() const { return t == 0; }
+  __device__ bool last() const { return t + 1 == spg; }
+};
+
 // kMode 0: write int32 accumulators acc[g,m,n].  kMode 1: write y (Eq. 11).
 template <int kMode, typename TY>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
@@ -124,7 +139,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  SharedCtl* ctl = reinterpret_cast<SharedCtl*>(smem + (size_t)kStages * kStageBytes);
+  SharedCtl* ctl = reinterpret_cast<SharedCtl*>(smem + (size_t)kSlots * kSlotBytes);
   volatile int* abort_flag = &ctl->abort_flag;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_rank();
@@ -138,11 +153,11 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
   const int64_t w_blocks_k = (a.K + 127) / 128;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) {
-      // rank 0's full barrier collects, per stage: its own TMA (1 arrival + the bytes), rank 1's
-      // "codes landed" (1) and the expander warps of both CTAs (2 x 4), so the MMA issuer makes
-      // one wait per stage.  Rank 1's copy only tracks its own TMA.
-      mbar_init(smem_u32(&ctl->full[s]), leader ? 2 + 2 * (kHalfN / 32) : 1);
+    for (int s = 0; s < kSlots; ++s) {
+      // rank 0's full barrier collects, per slot: its own TMA (1 arrival + the bytes), rank 1's
+      // "codes landed" (1) and the expander warps of both CTAs (2 CTAs x kGroups x 4), so the MMA
+      // issuer makes one wait per slot.  Rank 1's copy only tracks its own TMA.
+      mbar_init(smem_u32(&ctl->full[s]), leader ? 2 + 2 * kGroups * (kHalfN / 32) : 1);
       mbar_init(smem_u32(&ctl->empty[s]), 1);
     }
     for (int b = 0; b < 2; ++b) {
@@ -166,133 +181,122 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer (own codes)
     if (lane == 0) {
-      int stage = 0; uint32_t phase = 0;
+      int slot = 0; uint32_t phase = 0;
       uint32_t issued = 0;
-      bool ok = true;
-      for (PairIter it(tiles, m_tiles); ok && it.valid(); it.next()) {
-        const int m0 = (int)(it.m_tile() * kPairM + rank * kBM);
-        for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!mbar_wait2(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
-          const uint32_t bar = smem_u32(&ctl->full[stage]);
-          mbar_arrive_expect_tx(bar, (uint32_t)tx_bytes);
-          tma_load_2d(smem_u32(smem + (size_t)stage * kStageBytes), &map_x, kb * kBK, m0, bar);
-          ++issued;
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
-        }
+      for (StepIter st(tiles, m_tiles, a.G, kb_per_group); st.valid(); st.next()) {
+        const int m0 = (int)(st.it.m_tile() * kPairM + rank * kBM);
+        if (!mbar_wait2(smem_u32(&ctl->empty[slot]), phase ^ 1u, abort_flag)) break;
+        const uint32_t bar = smem_u32(&ctl->full[slot]);
+        const int nblk = st.nblk();
+        mbar_arrive_expect_tx(bar, (uint32_t)(tx_bytes * nblk));
+        for (int j = 0; j < nblk; ++j)
+          tma_load_2d(smem_u32(smem + (size_t)slot * kSlotBytes + (size_t)j * kStageBytes), &map_x,
+                      (st.kb0() + j) * kBK, m0, bar);
+        ++issued;
+        if (++slot == kSlots) { slot = 0; phase ^= 1u; }
       }
       // copies still in flight must land before the CTA may exit (bounded)
-      const uint32_t pending = issued < (uint32_t)kStages ? issued : (uint32_t)kStages;
+      const uint32_t pending = issued < (uint32_t)kSlots ? issued : (uint32_t)kSlots;
       for (uint32_t i = 0; i < pending; ++i) {
-        if (stage == 0) { stage = kStages; phase ^= 1u; }
-        --stage;
-        (void)mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag);
+        if (slot == 0) { slot = kSlots; phase ^= 1u; }
+        --slot;
+        (void)mbar_wait(smem_u32(&ctl->full[slot]), phase, abort_flag);
       }
     }
   } else if (warp == 1 && !leader) {
     // ---------------------------------------------------------------- rank 1: codes-landed forwarder
     if (lane == 0) {
-      int stage = 0; uint32_t phase = 0;
-      bool ok = true;
-      for (PairIter it(tiles, m_tiles); ok && it.valid(); it.next()) {
-        for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
-          mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->full[stage]), 0));
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
-        }
+      int slot = 0; uint32_t phase = 0;
+      for (StepIter st(tiles, m_tiles, a.G, kb_per_group); st.valid(); st.next()) {
+        if (!mbar_wait(smem_u32(&ctl->full[slot]), phase, abort_flag)) break;
+        mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->full[slot]), 0));
+        if (++slot == kSlots) { slot = 0; phase ^= 1u; }
       }
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- rank 0: MMA issuer for the pair
     if (lane == 0) {
-      int stage = 0; uint32_t phase = 0;
+      int slot = 0; uint32_t phase = 0;
       uint32_t pass = 0;
-      bool ok = true;
+      uint32_t d_tmem = tmem_base, buf = 0;
       const uint32_t empty0 = map_to_rank(smem_u32(&ctl->empty[0]), 0), empty1 = map_to_rank(smem_u32(&ctl->empty[0]), 1);
-      for (PairIter it(tiles, m_tiles); ok && it.valid(); it.next()) {
-        for (int g = 0; ok && g < a.G; ++g, ++pass) {
-          const uint32_t buf = pass & 1u, acc_phase = (pass >> 1) & 1u;
-          if (!mbar_wait2(smem_u32(&ctl->tmem_empty[buf]), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+      const uint32_t tfull0 = map_to_rank(smem_u32(&ctl->tmem_full[0]), 0), tfull1 = map_to_rank(smem_u32(&ctl->tmem_full[0]), 1);
+      for (StepIter st(tiles, m_tiles, a.G, kb_per_group); st.valid(); st.next()) {
+        if (st.first()) {                                      // a new (tile, group): next accumulator
+          buf = pass & 1u;
+          const uint32_t acc_phase = (pass >> 1) & 1u;
+          if (!mbar_wait2(smem_u32(&ctl->tmem_empty[buf]), acc_phase ^ 1u, abort_flag)) break;
           tc_fence_after();
-          const uint32_t d_tmem = tmem_base + buf * (uint32_t)kBN;
-          for (int kb = 0; kb < kb_per_group; ++kb) {
-            if (!mbar_wait2(smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t a_addr = smem_u32(smem + (size_t)stage * kStageBytes);
-            const uint64_t adesc = smem_desc_sw128(a_addr);
-            const uint64_t bdesc = smem_desc_sw128(a_addr + kABytes);
+          d_tmem = tmem_base + buf * (uint32_t)kBN;
+        }
+        if (!mbar_wait2(smem_u32(&ctl->full[slot]), phase, abort_flag)) break;
+        tc_fence_after();
+        const uint32_t a_addr = smem_u32(smem + (size_t)slot * kSlotBytes);
+        const int nblk = st.nblk();
+        for (int b = 0; b < nblk; ++b) {
+          const uint64_t adesc = smem_desc_sw128(a_addr + (uint32_t)b * kStageBytes);
+          const uint64_t bdesc = smem_desc_sw128(a_addr + (uint32_t)b * kStageBytes + kABytes);
 #pragma unroll
-            for (int j = 0; j < kBK / 32; ++j)
-              mma_i8_pair(d_tmem, adesc + (uint64_t)(2 * j), bdesc + (uint64_t)(2 * j), kIdesc,
-                          (kb > 0 || j > 0) ? 1u : 0u);
-            mma_commit_pair(empty0 + 8u * (uint32_t)stage);
-            mma_commit_pair(empty1 + 8u * (uint32_t)stage);
-            if (++stage == kStages) { stage = 0; phase ^= 1u; }
-          }
-          if (ok) {
-            const uint32_t f = smem_u32(&ctl->tmem_full[buf]);
-            mma_commit_pair(map_to_rank(f, 0));
-            mma_commit_pair(map_to_rank(f, 1));
-          }
+          for (int j = 0; j < kBK / 32; ++j)
+            mma_i8_pair(d_tmem, adesc + (uint64_t)(2 * j), bdesc + (uint64_t)(2 * j), kIdesc,
+                        (!st.first() || b > 0 || j > 0) ? 1u : 0u);
+        }
+        mma_commit_pair(empty0 + 8u * (uint32_t)slot);
+        mma_commit_pair(empty1 + 8u * (uint32_t)slot);
+        if (++slot == kSlots) { slot = 0; phase ^= 1u; }
+        if (st.last()) {                                       // accumulator of this (tile, group) complete
+          mma_commit_pair(tfull0 + 8u * buf);
+          mma_commit_pair(tfull1 + 8u * buf);
+          ++pass;
         }
       }
     }
   } else if (warp >= kExpandWarp0) {
     // ---------------------------------------------------------------- weight expanders (own half of B)
-    const int eg = (warp - kExpandWarp0) >> 2;                       // group number
+    const int eg = (warp - kExpandWarp0) >> 2;                       // group: fills k-block eg of every slot
     const int u = (threadIdx.x - kExpandWarp0 * 32) & (kHalfN - 1);  // row of this CTA's half, 0..127
-    const uint32_t row_base = smem_u32(smem) + (uint32_t)kABytes + (uint32_t)u * 128u + ((uint32_t)(u & 7) << 4);
-    int stage = eg; uint32_t phase = 0;
+    const uint32_t row_base = smem_u32(smem) + (uint32_t)eg * kStageBytes + (uint32_t)kABytes + (uint32_t)u * 128u +
+                              ((uint32_t)(u & 7) << 4);
+    int slot = 0; uint32_t phase = 0;
     const uint32_t full0 = map_to_rank(smem_u32(&ctl->full[0]), 0);
-    PairIter pf_it(tiles, m_tiles);
-    int pf_kb = eg;
-    const uint8_t* pf_src = nullptr;                                 // row u of the tile's first k-block
-    auto seek = [&]() {
-      while (pf_it.valid() && pf_kb >= k_blocks) { pf_kb -= k_blocks; pf_it.next(); }
-      pf_src = nullptr;
-      if (pf_it.valid()) {
-        const int64_t nb = (int64_t)pf_it.n_tile() * 2 + rank;
-        if (nb < w_blocks_n) pf_src = a.W_packed + nb * w_blocks_k * 2048 + u * 16;
-      }
-    };
-    seek();
+    // the 16 bytes of sign bits of the next two steps are prefetched in registers
+    StepIter pf(tiles, m_tiles, a.G, kb_per_group);
     auto fetch = [&]() -> uint4 {
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (pf_it.valid()) {
-        if (pf_src) v = __ldg(reinterpret_cast<const uint4*>(pf_src + (size_t)pf_kb * 2048));
-        pf_kb += kGroups;
-        if (pf_kb >= k_blocks) seek();
+      if (pf.valid()) {
+        const int64_t nb = (int64_t)pf.it.n_tile() * 2 + rank;
+        if (eg < pf.nblk() && nb < w_blocks_n)
+          v = __ldg(reinterpret_cast<const uint4*>(a.W_packed + (nb * w_blocks_k + pf.kb0() + eg) * 2048 + u * 16));
+        pf.next();
       }
       return v;
     };
     uint4 b0 = fetch(), b1 = fetch();
-    const uint32_t nclusters = gridDim.x >> 1, cid = blockIdx.x >> 1;
-    const uint32_t my_tiles = (tiles > cid) ? (tiles - cid + nclusters - 1) / nclusters : 0u;
-    const uint64_t flat = (uint64_t)my_tiles * (uint64_t)k_blocks;
-    const uint64_t owned = flat > (uint64_t)eg ? (flat - eg + kGroups - 1) / kGroups : 0;
-    for (uint64_t i = 0; i < owned; ++i) {
+    for (StepIter st(tiles, m_tiles, a.G, kb_per_group); st.valid(); st.next()) {
       const uint4 cur = b0;
       b0 = b1;
       b1 = fetch();
       bool got = true;
-      if (lane == 0) got = mbar_wait2(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag);
+      if (lane == 0) got = mbar_wait2(smem_u32(&ctl->empty[slot]), phase ^ 1u, abort_flag);
       got = __shfl_sync(0xFFFFFFFFu, got, 0);
       __syncwarp();
       if (!got) break;
-      const uint32_t dst = row_base + (uint32_t)stage * (uint32_t)kStageBytes;
-      const uint32_t words[4] = {cur.x, cur.y, cur.z, cur.w};
+      if (eg < st.nblk()) {
+        const uint32_t dst = row_base + (uint32_t)slot * (uint32_t)kSlotBytes;
+        const uint32_t words[4] = {cur.x, cur.y, cur.z, cur.w};
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        const uint32_t wd = words[c >> 1];
-        const int j0 = (c & 1) * 4;
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst ^ ((uint32_t)c << 4)),
-                     "r"(signs4(wd, j0)), "r"(signs4(wd, j0 + 1)), "r"(signs4(wd, j0 + 2)),
-                     "r"(signs4(wd, j0 + 3)) : "memory");
+        for (int c = 0; c < 8; ++c) {
+          const uint32_t wd = words[c >> 1];
+          const int j0 = (c & 1) * 4;
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst ^ ((uint32_t)c << 4)),
+                       "r"(signs4(wd, j0)), "r"(signs4(wd, j0 + 1)), "r"(signs4(wd, j0 + 2)),
+                       "r"(signs4(wd, j0 + 3)) : "memory");
+        }
+        fence_proxy_async_smem();
       }
-      fence_proxy_async_smem();
       __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(full0 + 8u * (uint32_t)stage);
-      stage += kGroups;
-      if (stage >= kStages) { stage -= kStages; phase ^= 1u; }
+      if (lane == 0) mbar_arrive_cluster(full0 + 8u * (uint32_t)slot);
+      if (++slot == kSlots) { slot = 0; phase ^= 1u; }
     }
   } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + 4) {
     // ---------------------------------------------------------------- epilogue (own 128 tokens)
