@@ -355,7 +355,7 @@ rows_per_token(const T* __restrict__ x, int64_t segments, int64_t K, int G, int 
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kRowWarps * 32, 2)
+__global__ void __launch_bounds__(kRowWarps * 32, 3)
 rows_tensor_stats(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg, float ln_eps, double inv_kg,
                   TensorScope* sc, SegRecord* __restrict__ recs) {
   const int lane = threadIdx.x & 31;
