@@ -155,7 +155,8 @@ bl_status bitlinear_matmul_i32(const int8_t* x_q, int64_t M, int64_t K, int64_t 
   if (!ws || ws_bytes < gemm_ws_total(M, N, G)) return BL_ERR_WORKSPACE;
   if (!aligned16(ws)) return BL_ERR_ALIGN;
   cudaStream_t s = (cudaStream_t)stream;
-  if (cudaMemsetAsync(ws, 0, kStatusBytes, s) != cudaSuccess) return BL_ERR_CUDA;
+  // the tensor-core kernel clears the status word itself; the CUDA-core kernel never writes it
+  if (layout != BL_LAYOUT_PREFILL && cudaMemsetAsync(ws, 0, kStatusBytes, s) != cudaSuccess) return BL_ERR_CUDA;
   GemmArgs a{};
   a.x_q = x_q; a.M = M; a.K = K; a.N = N; a.G = G; a.W_packed = W_packed; a.acc = acc;
   a.y = nullptr; a.gran = BL_PER_TENSOR; a.status = reinterpret_cast<uint32_t*>(ws);
@@ -182,7 +183,8 @@ bl_status bitlinear_matmul_dequant(const int8_t* x_q, int64_t M, int64_t K, int6
   if (!ws || ws_bytes < gemm_ws_total(M, N, G)) return BL_ERR_WORKSPACE;
   if (!aligned16(ws)) return BL_ERR_ALIGN;
   cudaStream_t s = (cudaStream_t)stream;
-  if (cudaMemsetAsync(ws, 0, kStatusBytes, s) != cudaSuccess) return BL_ERR_CUDA;
+  // the tensor-core kernel clears the status word itself; the CUDA-core kernel never writes it
+  if (layout != BL_LAYOUT_PREFILL && cudaMemsetAsync(ws, 0, kStatusBytes, s) != cudaSuccess) return BL_ERR_CUDA;
   GemmArgs a{};
   a.x_q = x_q; a.M = M; a.K = K; a.N = N; a.G = G; a.W_packed = W_packed; a.acc = nullptr;
   a.y = y; a.yt = yt; a.beta = beta; a.gamma = gamma; a.eta = eta; a.gran = gran;
@@ -216,7 +218,8 @@ bl_status bitlinear_forward(const void* x, bl_dtype xt, int64_t M, int64_t K, in
   if (!aligned16(ws)) return BL_ERR_ALIGN;
   char* base = reinterpret_cast<char*>(ws);
   cudaStream_t s = (cudaStream_t)stream;
-  if (cudaMemsetAsync(base + w.status, 0, kStatusBytes, s) != cudaSuccess) return BL_ERR_CUDA;
+  if (layout != BL_LAYOUT_PREFILL && cudaMemsetAsync(base + w.status, 0, kStatusBytes, s) != cudaSuccess)
+    return BL_ERR_CUDA;
   int8_t* codes = reinterpret_cast<int8_t*>(base + w.codes);
   float* gamma = reinterpret_cast<float*>(base + w.gamma);
   float* eta = reinterpret_cast<float*>(base + w.eta);

@@ -165,6 +165,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
       mbar_init(smem_u32(&ctl->tmem_empty[b]), 8);
     }
     ctl->abort_flag = 0;
+    if (blockIdx.x == 0) *a.status = 0u;             // a timeout (seconds later) overwrites it
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 2) {
