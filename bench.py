@@ -119,8 +119,17 @@ class ClockSampler:
             return dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0, source="unavailable")
 
 
-def event_pairs_ms(pairs):
-    return [a.elapsed_time(b) for a, b in pairs]
+def job_throughput(units_local, ms_local, dist=None, device=None):
+    """Whole-job rate of replicas that each processed `units_local` units in `ms_local` ms: the sum
+    of the units over the ranks divided by the slowest rank's time.  Returns (units per second,
+    max ms).  `dist` is torch.distributed (any backend) or None for one process."""
+    if dist is None:
+        return units_local / (ms_local * 1e-3), ms_local
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    u = torch.tensor([units_local], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(u.item()) / (float(t.item()) * 1e-3), float(t.item())
 
 
 # --------------------------------------------------------------------------------------- own arm
@@ -149,13 +158,6 @@ def run_b200(args):
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
-
-    def max_over_ranks(ms):
-        if dist is None:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
 
     # ---- prefill workload: inputs resident in HBM, ROTATE distinct sets (> L2 in total) ----------
     M, K, N, G = PREFILL["M"], PREFILL["K"], PREFILL["N"], PREFILL["G"]
@@ -196,11 +198,11 @@ def run_b200(args):
             step(i, evs[i])
         t1.record()
         barrier()
-    total_ms = max_over_ranks(t0.elapsed_time(t1))
+    ops_per_step = 2.0 * M * N * K
+    job_ops_per_s, total_ms = job_throughput(ops_per_step * K_steps, t0.elapsed_time(t1), dist, dev)
     assert B.ws_status(ws_g) == B.OK
     ms_per_step = total_ms / K_steps
-    ops_per_step = 2.0 * M * N * K
-    value = world * ops_per_step / (ms_per_step * 1e-3) / 1e12
+    value = job_ops_per_s / 1e12
     gemm_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
     quant_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
     gemm_tops = ops_per_step / (gemm_ms * 1e-3) / 1e12
@@ -228,8 +230,9 @@ def run_b200(args):
         e2e_step(i)
     t1.record()
     barrier()
-    e2e_ms = max_over_ranks(t0.elapsed_time(t1)) / e2e_steps
-    e2e = dict(value=world * ops_per_step / (e2e_ms * 1e-3) / 1e12, unit="TOPS", ms_per_step=e2e_ms,
+    e2e_ops_per_s, e2e_total = job_throughput(ops_per_step * e2e_steps, t0.elapsed_time(t1), dist, dev)
+    e2e_ms = e2e_total / e2e_steps
+    e2e = dict(value=e2e_ops_per_s / 1e12, unit="TOPS", ms_per_step=e2e_ms,
                h2d_bytes_per_step=M * K * 2, d2h_bytes_per_step=M * N * 2,
                call="bitlinear_forward on device copies of pinned host x; y copied back to pinned host")
 
