@@ -377,7 +377,7 @@ def bench_pack(B, synth, dev, peaks):
     nbytes = 2.0 * N * K * 4 + N * K / 8
     gbs = nbytes / (ms * 1e-3) / 1e9
     return {"workload": "binarize+pack W fp32 [4096,4096] -> 1 bit/weight (PREFILL layout), alpha, beta, rowsum",
-            "ms": ms, "gpu_launches": 3 * reps,
+            "ms": ms, "gpu_launches": 2 * reps,
             "roofline": {"bound": "hbm", "kernel": "reduce_partials + sign_pack", "achieved": gbs,
                          "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": None,
                          "peak_source": peaks["source"] + " copy"}}
