@@ -12,8 +12,7 @@
 //
 // Roles per CTA:
 //   warp 0      TMA producer for this CTA's codes tile
-//   warp 1      rank 0: MMA issuer for the pair (one thread); rank 1: forwards "my codes tile has
-//               landed" to rank 0's barrier
+//   warp 1      rank 0: MMA issuer for the pair (one thread); idle in rank 1
 //   warp 2      tensor-memory allocation (both CTAs, cta_group::2)
 //   warps 4-7   epilogue
 //   warps 8-15  weight expanders: two groups of 4 warps, group e fills k-block e of every ring slot;
@@ -21,11 +20,11 @@
 // A ring slot holds two k-blocks (256 weights): the MMA issuer, whose serial work per barrier round
 // trip bounds the kernel, waits and commits once per slot and issues 8 MMAs in between.
 // Barriers.  In every CTA: empty (stage consumed; the issuer commits to both CTAs' copies) and
-// tmem_full (accumulator complete; committed to both).  full: in rank 0 one barrier per slot
-// collects its own TMA bytes, rank 1's "codes landed" and the 8 expander warps of the pair, so the
-// issuer waits once per slot; in rank 1
-// it tracks that CTA's TMA only.  tmem_empty (rank 0) takes the 8 epilogue warps of the pair.
-// Remote arrivals are mbarrier.arrive on the mapa address of rank 0's barrier.
+// tmem_full (accumulator complete; committed to both).  full (rank 0 only): one barrier per slot
+// collects the TMA bytes of both CTAs' codes tiles (rank 1's copies complete on rank 0's barrier:
+// cp.async.bulk.tensor.cta_group::2) and the expander warps of the pair, so the issuer waits once
+// per slot.  tmem_empty (rank 0) takes the 8 epilogue warps of the pair.  Remote arrivals are
+// mbarrier.arrive on the mapa address of rank 0's barrier.
 //
 // Every wait is bounded; a limit that runs out raises the CTA's abort flag, records
 // BL_ERR_TIMEOUT and lets every role fall through to the common exit (cluster barrier, tensor
@@ -91,6 +90,18 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
 __device__ __forceinline__ bool mbar_wait2(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   return mbar_wait(bar, parity, abort_flag);
 }
+// TMA tile load whose completion bytes are counted on a barrier that may live in the partner CTA
+// (the destination is always this CTA's shared memory).  No multicast.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1,
+                                                 uint32_t bar_cluster_addr) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar_cluster_addr) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx_cluster(uint32_t bar_cluster_addr, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(bar_cluster_addr), "r"(bytes)
+               : "memory");
+}
 __device__ __forceinline__ void mma_i8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                             uint32_t accumulate) {
   asm volatile(
@@ -154,10 +165,10 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kSlots; ++s) {
-      // rank 0's full barrier collects, per slot: its own TMA (1 arrival + the bytes), rank 1's
-      // "codes landed" (1) and the expander warps of both CTAs (2 CTAs x kGroups x 4), so the MMA
-      // issuer makes one wait per slot.  Rank 1's copy only tracks its own TMA.
-      mbar_init(smem_u32(&ctl->full[s]), leader ? 2 + 2 * kGroups * (kHalfN / 32) : 1);
+      // rank 0's full barrier collects, per slot: the TMA producers of both CTAs (1 arrival each,
+      // plus the bytes of both codes tiles) and the expander warps of both CTAs (2 x kGroups x 4),
+      // so the MMA issuer makes one wait per slot.  Rank 1's copy is unused.
+      mbar_init(smem_u32(&ctl->full[s]), 2 + 2 * kGroups * (kHalfN / 32));
       mbar_init(smem_u32(&ctl->empty[s]), 1);
     }
     for (int b = 0; b < 2; ++b) {
@@ -183,40 +194,24 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
     // ---------------------------------------------------------------- TMA producer (own codes)
     if (lane == 0) {
       int slot = 0; uint32_t phase = 0;
-      uint32_t issued = 0;
+      const uint32_t full0 = map_to_rank(smem_u32(&ctl->full[0]), 0);      // both CTAs report to rank 0
       for (StepIter st(tiles, m_tiles, a.G, kb_per_group); st.valid(); st.next()) {
         const int m0 = (int)(st.it.m_tile() * kPairM + rank * kBM);
         if (!mbar_wait2(smem_u32(&ctl->empty[slot]), phase ^ 1u, abort_flag)) break;
-        const uint32_t bar = smem_u32(&ctl->full[slot]);
+        const uint32_t bar = full0 + 8u * (uint32_t)slot;
         const int nblk = st.nblk();
-        mbar_arrive_expect_tx(bar, (uint32_t)(tx_bytes * nblk));
+        mbar_arrive_expect_tx_cluster(bar, (uint32_t)(tx_bytes * nblk));
         for (int j = 0; j < nblk; ++j)
-          tma_load_2d(smem_u32(smem + (size_t)slot * kSlotBytes + (size_t)j * kStageBytes), &map_x,
-                      (st.kb0() + j) * kBK, m0, bar);
-        ++issued;
+          tma_load_2d_pair(smem_u32(smem + (size_t)slot * kSlotBytes + (size_t)j * kStageBytes), &map_x,
+                           (st.kb0() + j) * kBK, m0, bar);
         if (++slot == kSlots) { slot = 0; phase ^= 1u; }
       }
-      // copies still in flight must land before the CTA may exit (bounded)
-      const uint32_t pending = issued < (uint32_t)kSlots ? issued : (uint32_t)kSlots;
-      for (uint32_t i = 0; i < pending; ++i) {
-        if (slot == 0) { slot = kSlots; phase ^= 1u; }
-        --slot;
-        (void)mbar_wait(smem_u32(&ctl->full[slot]), phase, abort_flag);
-      }
-    }
-  } else if (warp == 1 && !leader) {
-    // ---------------------------------------------------------------- rank 1: codes-landed forwarder
-    if (lane == 0) {
-      int slot = 0; uint32_t phase = 0;
-      for (StepIter st(tiles, m_tiles, a.G, kb_per_group); st.valid(); st.next()) {
-        if (!mbar_wait(smem_u32(&ctl->full[slot]), phase, abort_flag)) break;
-        mbar_arrive_cluster(map_to_rank(smem_u32(&ctl->full[slot]), 0));
-        if (++slot == kSlots) { slot = 0; phase ^= 1u; }
-      }
+      // Every copy issued here is consumed by an MMA before the accumulator it feeds is released,
+      // and the epilogue warps of this CTA wait for that release: no copy is in flight at exit.
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- rank 0: MMA issuer for the pair
-    if (lane == 0) {
+    if (lane == 0 && leader) {
       int slot = 0; uint32_t phase = 0;
       uint32_t pass = 0;
       uint32_t d_tmem = tmem_base, buf = 0;
