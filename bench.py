@@ -35,6 +35,15 @@ ROTATE = 3                                           # distinct input/output set
 NOMINAL_INT8_TOPS = 4500.0
 NOMINAL_HBM_GBS = 8000.0
 INT8_TO_BF16 = 2.0                                   # nominal dense int8 : bf16 tensor rate
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the summaries under
+# profiles/, taken with ncu on these same workloads.  A figure is valid only while its kernel is the
+# one that was profiled: set it to None when the kernel changes, until the capture is redone.
+NCU_TRAFFIC = {
+    "gemm_tc2_kernel": 54.1e6,                       # 36.3 MB read + 17.8 MB written (y largely still in L2)
+    "rows_tensor_stats + rows_tensor_codes": 140.3e6,   # 67.1 + 0.5 and 67.4 + 5.4 MB
+    "gemv_decode_kernel": 8.45e6,
+    "reduce_partials + sign_pack": 135.3e6,          # 67.1 + 0.4 and 67.1 + 0.7 MB
+}
 
 
 def load_peaks():
@@ -251,14 +260,14 @@ def run_b200(args):
         "gpu_launches": 4 * K_steps,
         "kernels_per_step": ["init_scope", "rows_tensor_stats", "rows_tensor_codes", "gemm_tc2_kernel"],
         "roofline": {"bound": "tensor", "kernel": "gemm_tc2_kernel", "achieved": gemm_tops, "peak": tensor_peak,
-                     "unit": "TFLOP/s", "frac": gemm_tops / tensor_peak, "traffic": None,
+                     "unit": "TFLOP/s", "frac": gemm_tops / tensor_peak, "traffic": NCU_TRAFFIC["gemm_tc2_kernel"],
                      "op_kind": "int8 (s8 x s8 -> s32), 2 ops per multiply-accumulate",
                      "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} x {INT8_TO_BF16} "
                                     "(nominal int8:bf16 ratio)",
                      "frac_of_nominal": gemm_tops / NOMINAL_INT8_TOPS, "avg_launch_ms": gemm_ms},
         "roofline_quant": {"bound": "hbm", "kernel": "rows_tensor_stats + rows_tensor_codes", "achieved": quant_gbs,
                            "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": quant_gbs / peaks["hbm_gbs"],
-                           "traffic": None, "avg_ms": quant_ms, "peak_source": peaks["source"] + " copy"},
+                           "traffic": NCU_TRAFFIC["rows_tensor_stats + rows_tensor_codes"], "avg_ms": quant_ms, "peak_source": peaks["source"] + " copy"},
     }
 
     parts = set(args.parts.split(","))
@@ -353,7 +362,7 @@ def bench_decode(B, synth, dev, peaks):
                 "frac_2": rate(out["hbm_2streams"]) / peaks["hbm_gbs"],
                 "frac_4": rate(out["hbm_4streams"]) / peaks["hbm_gbs"]},
             "roofline": {"bound": "hbm", "kernel": "gemv_decode_kernel", "achieved": gbs, "peak": peaks["hbm_gbs"],
-                         "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": None,
+                         "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC["gemv_decode_kernel"],
                          "frac_of_nominal": gbs / NOMINAL_HBM_GBS, "peak_source": peaks["source"] + " copy"}}
 
 
@@ -379,7 +388,8 @@ def bench_pack(B, synth, dev, peaks):
     return {"workload": "binarize+pack W fp32 [4096,4096] -> 1 bit/weight (PREFILL layout), alpha, beta, rowsum",
             "ms": ms, "gpu_launches": 2 * reps,
             "roofline": {"bound": "hbm", "kernel": "reduce_partials + sign_pack", "achieved": gbs,
-                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": None,
+                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                         "traffic": NCU_TRAFFIC["reduce_partials + sign_pack"],
                          "peak_source": peaks["source"] + " copy"}}
 
 
