@@ -74,7 +74,8 @@ typedef enum {
   BL_OP_QUANT_ACT = 1,
   BL_OP_FORWARD = 2,
   BL_OP_MATMUL_I32 = 3,
-  BL_OP_MATMUL_DEQUANT = 4
+  BL_OP_MATMUL_DEQUANT = 4,
+  BL_OP_BLOCK_FORWARD = 5    /* M = batch * seq tokens, N = ffn width, K = model width d, G ignored (1) */
 } bl_op;
 
 /* Human-readable name of a status code (static string, never NULL). */
@@ -184,6 +185,41 @@ bl_status bitlinear_gemv_decode(const void* x, bl_dtype xt, int64_t K, int64_t N
                                 bl_quant_mode mode, float ln_eps, int eta_correction,
                                 const uint8_t* W_packed, const float* beta,
                                 const int32_t* rowsum, void* y, bl_dtype yt, void* stream);
+
+/* Causal self-attention core of the decoder block (Sec. 2, Fig. 2b; the paper keeps it in high
+ * precision): per batch and head O = softmax(Q K^T / sqrt(d_h) + causal mask) V, fp16 in and out,
+ * fp32 softmax statistics and accumulators.  No positional encoding.
+ *   q, k, v  fp16 [batch*seq, heads*128] with a common row stride ld (elements), so they may be
+ *            column blocks of one buffer;  o fp16, same shape, row stride ld_o.
+ *   head_dim must be 128, seq a multiple of 64, ld and ld_o multiples of 8. */
+bl_status bitlinear_attention_causal(const void* q, const void* k, const void* v, void* o, int batch, int seq,
+                                     int heads, int head_dim, int64_t ld, int64_t ld_o, void* stream);
+
+/* One BitNet decoder block, forward (Sec. 2, Fig. 2b): every linear map is a BitLinear (its own
+ * LN + per-token 8-bit quantisation in front, Eq. 11), the attention core and the residual adds
+ * stay in fp16:
+ *     q, k, v = BitLinear_{Q,K,V}(x)            (one LN + quant of x feeds all three)
+ *     a       = causal attention(q, k, v)
+ *     h       = x + BitLinear_O(a)
+ *     u       = ReLU(BitLinear_up(h))
+ *     y       = h + BitLinear_down(u)           (down uses the eta form of Eq. 6 on its input)
+ * d = heads * 128; FFN width ffn; tokens T = batch * seq (seq % 64 == 0); d % 128 == 0, ffn % 128 == 0.
+ * All weight buffers are PREFILL-packed with one group: W_q, W_k, W_v, W_o [d,d], W_up [ffn,d],
+ * W_down [d,ffn]; beta_* point to one float each (as written by bitlinear_binarize_pack).
+ * Every intermediate is a caller buffer (fp16, row-major), so each stage can be inspected:
+ *   q, k, v, a, h [T,d];  u [T,ffn];  y [T,d] (also used for the two projection outputs).
+ * Workspace: BL_OP_BLOCK_FORWARD (codes, gamma, eta, quant and GEMM scratch).  Asynchronous on
+ * `stream`; bitlinear_ws_status(ws, stream) reports a device-side timeout of the GEMMs. */
+typedef struct {
+  const uint8_t *W_q, *W_k, *W_v, *W_o, *W_up, *W_down;
+  const float *beta_q, *beta_k, *beta_v, *beta_o, *beta_up, *beta_down;
+} bl_block_weights;
+typedef struct {
+  void *q, *k, *v, *a, *h, *u;
+} bl_block_buffers;
+bl_status bitlinear_block_forward(const void* x, int batch, int seq, int heads, int64_t ffn, float ln_eps,
+                                  const bl_block_weights* w, const bl_block_buffers* buf, void* y, void* ws,
+                                  size_t ws_bytes, void* stream);
 
 /* Synchronises `stream`, then reads the status word a previous bitlinear_forward or
  * bitlinear_matmul_i32 call left in `ws`.  BL_OK, BL_ERR_TIMEOUT, or BL_ERR_CUDA. */

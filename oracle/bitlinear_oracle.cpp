@@ -267,4 +267,44 @@ int oracle_forward(const float* x, int64_t M, int64_t K, int64_t N, int G, int m
   return 0;
 }
 
+
+// Causal self-attention core of the decoder block (Sec. 2, Fig. 2b), written out from its
+// definition in double precision: for query t of (batch b, head h)
+//   o_t = sum_{s <= t} softmax_s(q_t . k_s / sqrt(d_h)) v_s .
+// q, k, v: float [batch*seq, heads*dh] row-major (values of the 16-bit inputs held exactly).
+// rows: `count` token indices (0 .. batch*seq-1) to evaluate, all heads each; out [count, heads*dh].
+int oracle_attention_rows(const float* q, const float* k, const float* v, int64_t batch, int64_t seq,
+                          int64_t heads, int64_t dh, const int64_t* rows, int64_t count, double* out) {
+  if (!q || !k || !v || !rows || !out || batch <= 0 || seq <= 0 || heads <= 0 || dh <= 0) return 1;
+  const int64_t ld = heads * dh;
+  const double scale = 1.0 / std::sqrt((double)dh);
+  for (int64_t i = 0; i < count; ++i)
+    if (rows[i] < 0 || rows[i] >= batch * seq) return 4;
+#pragma omp parallel for schedule(dynamic)
+  for (int64_t job = 0; job < count * heads; ++job) {
+    const int64_t i = job / heads, h = job % heads;
+    const int64_t tok = rows[i], b = tok / seq, t = tok % seq;
+    const float* qt = q + tok * ld + h * dh;
+    std::vector<double> score((size_t)(t + 1));
+    double mx = -std::numeric_limits<double>::infinity();
+    for (int64_t s = 0; s <= t; ++s) {                       // causal: keys 0..t of the same sequence
+      const float* ks = k + (b * seq + s) * ld + h * dh;
+      double dot = 0.0;
+      for (int64_t e = 0; e < dh; ++e) dot += (double)qt[e] * (double)ks[e];
+      score[(size_t)s] = dot * scale;
+      if (score[(size_t)s] > mx) mx = score[(size_t)s];
+    }
+    double denom = 0.0;
+    for (int64_t s = 0; s <= t; ++s) { score[(size_t)s] = std::exp(score[(size_t)s] - mx); denom += score[(size_t)s]; }
+    double* o = out + i * ld + h * dh;
+    for (int64_t e = 0; e < dh; ++e) o[e] = 0.0;
+    for (int64_t s = 0; s <= t; ++s) {
+      const float* vs = v + (b * seq + s) * ld + h * dh;
+      const double p = score[(size_t)s] / denom;
+      for (int64_t e = 0; e < dh; ++e) o[e] += p * (double)vs[e];
+    }
+  }
+  return 0;
+}
+
 }  // extern "C"

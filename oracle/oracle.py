@@ -144,3 +144,18 @@ def forward(x, bits, beta, G=1, mode=ABSMAX, gran=PER_TOKEN, ln_eps=1e-5, rowsum
     _check(rc, "forward")
     shape = (M, G) if gran == PER_TOKEN else (G,)
     return dict(y=y, codes=codes, gamma=gamma.reshape(shape), eta=eta.reshape(shape), acc=acc)
+
+
+def attention_rows(q, k, v, batch, seq, heads, dh, rows):
+    """Causal softmax(q k^T / sqrt(dh)) v (Sec. 2, Fig. 2b) in fp64 for the given token rows, all
+    heads.  q, k, v [batch*seq, heads*dh].  Returns f64 [len(rows), heads*dh]."""
+    q = np.ascontiguousarray(q, dtype=np.float32)
+    k = np.ascontiguousarray(k, dtype=np.float32)
+    v = np.ascontiguousarray(v, dtype=np.float32)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    out = np.zeros((len(rows), heads * dh), np.float64)
+    rc = lib().oracle_attention_rows(_p(q, C.c_float), _p(k, C.c_float), _p(v, C.c_float), C.c_int64(batch),
+                                     C.c_int64(seq), C.c_int64(heads), C.c_int64(dh), _p(rows, C.c_int64),
+                                     C.c_int64(len(rows)), _p(out, C.c_double))
+    _check(rc, "attention_rows")
+    return out

@@ -18,7 +18,7 @@ F32, F16, BF16 = 0, 1, 2
 ABSMAX, ETA = 0, 1
 PER_TENSOR, PER_TOKEN = 0, 1
 CANONICAL, PREFILL, DECODE = 0, 1, 2
-OP_BINARIZE_PACK, OP_QUANT_ACT, OP_FORWARD, OP_MATMUL_I32, OP_MATMUL_DEQUANT = 0, 1, 2, 3, 4
+OP_BINARIZE_PACK, OP_QUANT_ACT, OP_FORWARD, OP_MATMUL_I32, OP_MATMUL_DEQUANT, OP_BLOCK_FORWARD = 0, 1, 2, 3, 4, 5
 MAX_GROUPS = 64
 NOALLOC_MAX_SEGMENTS = 16384
 ERR_TOO_LARGE = 8
@@ -27,7 +27,7 @@ EXPORTS = [
     "bitlinear_status_string", "bitlinear_workspace_bytes", "bitlinear_packed_bytes",
     "bitlinear_layout_index", "bitlinear_binarize_pack", "bitlinear_quant_act", "bitlinear_quant_act_noalloc",
     "bitlinear_forward", "bitlinear_matmul_i32", "bitlinear_matmul_dequant", "bitlinear_gemv_decode",
-    "bitlinear_ws_status",
+    "bitlinear_attention_causal", "bitlinear_block_forward", "bitlinear_ws_status",
 ]
 
 _DTYPES = {torch.float32: F32, torch.float16: F16, torch.bfloat16: BF16}
@@ -74,6 +74,10 @@ def lib():
         L.bitlinear_gemv_decode.restype = ci
         L.bitlinear_gemv_decode.argtypes = [vp, ci, i64, i64, ci, ci, ci, C.c_float, ci, vp, vp, vp,
                                             vp, ci, vp]
+        L.bitlinear_attention_causal.restype = ci
+        L.bitlinear_attention_causal.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, i64, i64, vp]
+        L.bitlinear_block_forward.restype = ci
+        L.bitlinear_block_forward.argtypes = [vp, ci, ci, ci, i64, C.c_float, vp, vp, vp, vp, sz, vp]
         L.bitlinear_ws_status.restype = ci
         L.bitlinear_ws_status.argtypes = [vp, vp]
         _lib = L
@@ -234,6 +238,48 @@ def gemv_decode(x, W_packed, beta, N, G=1, mode=ABSMAX, ln_eps=1e-5, rowsum=None
                                        _ptr(rowsum), _ptr(y), _dt(y), _stream())
     _check(code, "bitlinear_gemv_decode")
     return y
+
+
+class _BlockWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("W_q", "W_k", "W_v", "W_o", "W_up", "W_down",
+                                          "beta_q", "beta_k", "beta_v", "beta_o", "beta_up", "beta_down")]
+
+
+class _BlockBuffers(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("q", "k", "v", "a", "h", "u")]
+
+
+def attention_causal(q, k, v, batch, seq, heads, head_dim=128, o=None):
+    """bitlinear_attention_causal.  q, k, v fp16 [batch*seq, heads*head_dim] (may be column slices of
+    one buffer with a common row stride); returns o fp16 [batch*seq, heads*head_dim]."""
+    T = batch * seq
+    if o is None:
+        o = torch.empty((T, heads * head_dim), dtype=torch.float16, device=q.device)
+    assert q.stride(1) == 1 and k.stride() == q.stride() and v.stride() == q.stride()
+    code = lib().bitlinear_attention_causal(_ptr(q), _ptr(k), _ptr(v), _ptr(o), batch, seq, heads, head_dim,
+                                            q.stride(0), o.stride(0), _stream())
+    _check(code, "bitlinear_attention_causal")
+    return o
+
+
+def block_forward(x, weights, batch, seq, heads, ffn, ln_eps=1e-5, ws=None):
+    """bitlinear_block_forward.  x fp16 [batch*seq, heads*128]; `weights` maps q, k, v, o, up, down to
+    the dicts returned by binarize_pack(layout=PREFILL).  Returns dict(y, q, k, v, a, h, u): the output
+    and every intermediate, all fp16."""
+    T, d = x.shape
+    dev = x.device
+    f16 = dict(dtype=torch.float16, device=dev)
+    out = {n: torch.empty((T, d), **f16) for n in ("q", "k", "v", "a", "h", "y")}
+    out["u"] = torch.empty((T, ffn), **f16)
+    w = _BlockWeights(*[weights[n]["W_packed"].data_ptr() for n in ("q", "k", "v", "o", "up", "down")],
+                      *[weights[n]["beta"].data_ptr() for n in ("q", "k", "v", "o", "up", "down")])
+    b = _BlockBuffers(*[out[n].data_ptr() for n in ("q", "k", "v", "a", "h", "u")])
+    ws = _ws(workspace_bytes(OP_BLOCK_FORWARD, T, ffn, d, 1), dev, ws)
+    code = lib().bitlinear_block_forward(_ptr(x), batch, seq, heads, ffn, float(ln_eps), C.byref(w), C.byref(b),
+                                         _ptr(out["y"]), _ptr(ws), ws.numel(), _stream())
+    _check(code, "bitlinear_block_forward")
+    out["ws"] = ws
+    return out
 
 
 def ws_status(ws) -> int:

@@ -25,6 +25,21 @@ size_t gemm_ws_total(int64_t M, int64_t N, int G) {
   return kStatusBytes + round256(gemm_tc_scratch_bytes(M, N, G));
 }
 
+struct BlockWs {                       // carving of the BL_OP_BLOCK_FORWARD workspace
+  size_t gemm, codes, gamma, eta, total;
+};
+BlockWs carve_block(int64_t T, int64_t d, int64_t ffn) {
+  BlockWs w;
+  size_t off = 0;
+  const int64_t widest = ffn > d ? ffn : d;
+  w.gemm = off;  off += gemm_ws_total(T, widest, 1);
+  w.codes = off; off += round256((size_t)T * (size_t)widest);
+  w.gamma = off; off += round256((size_t)T * sizeof(float));
+  w.eta = off;   off += round256((size_t)T * sizeof(float));
+  w.total = off;
+  return w;
+}
+
 struct ForwardWs {                     // carving of the BL_OP_FORWARD workspace
   size_t status, codes, gamma, eta, quant, total;
 };
@@ -73,6 +88,7 @@ size_t bitlinear_workspace_bytes(bl_op op, int64_t M, int64_t N, int64_t K, int 
     case BL_OP_FORWARD: return (M > 0 && N > 0) ? carve_forward(M, N, K, G).total : 0;
     case BL_OP_MATMUL_I32:
     case BL_OP_MATMUL_DEQUANT: return (M > 0 && N > 0) ? gemm_ws_total(M, N, G) : 0;
+    case BL_OP_BLOCK_FORWARD: return (M > 0 && N > 0) ? carve_block(M, K, N).total : 0;
   }
   return 0;
 }
@@ -252,6 +268,66 @@ bl_status bitlinear_gemv_decode(const void* x, bl_dtype xt, int64_t K, int64_t N
   if (!aligned16(x) || !aligned16(W_packed) || !aligned16(y)) return BL_ERR_ALIGN;
   GemvArgs a{x, xt, K, N, G, mode, ln_eps, eta_correction ? 1 : 0, W_packed, beta, rowsum, y, yt};
   return launch_gemv_decode(a, (cudaStream_t)stream) == cudaSuccess ? BL_OK : BL_ERR_CUDA;
+}
+
+bl_status bitlinear_attention_causal(const void* q, const void* k, const void* v, void* o, int batch, int seq,
+                                     int heads, int head_dim, int64_t ld, int64_t ld_o, void* stream) {
+  if (!q || !k || !v || !o) return BL_ERR_NULL;
+  if (batch <= 0 || seq <= 0 || heads <= 0 || seq % 64 != 0 || ld % 8 != 0 || ld_o % 8 != 0) return BL_ERR_SHAPE;
+  if (ld < (int64_t)heads * 128 || ld_o < (int64_t)heads * 128) return BL_ERR_SHAPE;
+  if (head_dim != 128) return BL_ERR_UNSUPPORTED;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return BL_ERR_ALIGN;
+  return launch_attention_causal(q, k, v, o, batch, seq, heads, ld, ld_o, (cudaStream_t)stream) == cudaSuccess
+             ? BL_OK : BL_ERR_CUDA;
+}
+
+bl_status bitlinear_block_forward(const void* x, int batch, int seq, int heads, int64_t ffn, float ln_eps,
+                                  const bl_block_weights* w, const bl_block_buffers* buf, void* y, void* ws,
+                                  size_t ws_bytes, void* stream) {
+  if (!x || !w || !buf || !y) return BL_ERR_NULL;
+  if (!w->W_q || !w->W_k || !w->W_v || !w->W_o || !w->W_up || !w->W_down) return BL_ERR_NULL;
+  if (!w->beta_q || !w->beta_k || !w->beta_v || !w->beta_o || !w->beta_up || !w->beta_down) return BL_ERR_NULL;
+  if (!buf->q || !buf->k || !buf->v || !buf->a || !buf->h || !buf->u) return BL_ERR_NULL;
+  if (batch <= 0 || seq <= 0 || heads <= 0 || ffn <= 0 || seq % 64 != 0 || ffn % 128 != 0) return BL_ERR_SHAPE;
+  const int64_t T = (int64_t)batch * seq, d = (int64_t)heads * 128;
+  if (!gemm_tc_supported(T, d, d, 1) || !gemm_tc_supported(T, d, ffn, 1) || !gemm_tc_supported(T, ffn, d, 1))
+    return BL_ERR_SHAPE;
+  const void* ptrs[] = {x, y, buf->q, buf->k, buf->v, buf->a, buf->h, buf->u, w->W_q, w->W_k, w->W_v, w->W_o,
+                        w->W_up, w->W_down};
+  for (const void* p : ptrs) if (!aligned16(p)) return BL_ERR_ALIGN;
+  const BlockWs c = carve_block(T, d, ffn);
+  if (!ws || ws_bytes < c.total) return BL_ERR_WORKSPACE;
+  if (!aligned16(ws)) return BL_ERR_ALIGN;
+  char* base = reinterpret_cast<char*>(ws);
+  cudaStream_t s = (cudaStream_t)stream;
+  int8_t* codes = reinterpret_cast<int8_t*>(base + c.codes);
+  float* gamma = reinterpret_cast<float*>(base + c.gamma);
+  float* eta = reinterpret_cast<float*>(base + c.eta);
+
+  // LN + per-token quantisation of `in` [T,K] (fp16), then W~ x~ rescaled into `out` [T,N] (fp16).
+  auto quant = [&](const void* in, int64_t K, bl_quant_mode mode) -> bool {
+    QuantArgs q{in, BL_F16, T, K, 1, mode, BL_PER_TOKEN, ln_eps, codes, gamma, eta, nullptr};
+    return launch_quant_act(q, s) == cudaSuccess;
+  };
+  auto matmul = [&](int64_t K, int64_t N, const uint8_t* W, const float* beta, void* out) -> bool {
+    GemmArgs g{};
+    g.x_q = codes; g.M = T; g.K = K; g.N = N; g.G = 1; g.W_packed = W; g.acc = nullptr; g.y = out; g.yt = BL_F16;
+    g.beta = beta; g.gamma = gamma; g.eta = eta; g.gran = BL_PER_TOKEN; g.rowsum = nullptr; g.eta_correction = 0;
+    g.status = reinterpret_cast<uint32_t*>(base + c.gemm);
+    g.scratch = base + c.gemm + kStatusBytes;
+    return launch_gemm_tc(g, s) == cudaSuccess;
+  };
+  bool ok = quant(x, d, BL_ABSMAX)
+      && matmul(d, d, w->W_q, w->beta_q, buf->q) && matmul(d, d, w->W_k, w->beta_k, buf->k)
+      && matmul(d, d, w->W_v, w->beta_v, buf->v)
+      && launch_attention_causal(buf->q, buf->k, buf->v, buf->a, batch, seq, heads, d, d, s) == cudaSuccess
+      && quant(buf->a, d, BL_ABSMAX) && matmul(d, d, w->W_o, w->beta_o, buf->h)
+      && launch_add_inplace(buf->h, x, T * d, s) == cudaSuccess
+      && quant(buf->h, d, BL_ABSMAX) && matmul(d, ffn, w->W_up, w->beta_up, buf->u)
+      && launch_relu_inplace(buf->u, T * ffn, s) == cudaSuccess
+      && quant(buf->u, ffn, BL_ETA) && matmul(ffn, d, w->W_down, w->beta_down, y)
+      && launch_add_inplace(y, buf->h, T * d, s) == cudaSuccess;
+  return ok ? BL_OK : BL_ERR_CUDA;
 }
 
 bl_status bitlinear_ws_status(const void* ws, void* stream) {

@@ -1,0 +1,194 @@
+// Causal self-attention core of the decoder block (Sec. 2, Fig. 2b): per batch and head,
+//   O = softmax(Q K^T / sqrt(d_h) + causal mask) V,
+// in fp16 with fp32 softmax statistics and accumulators.  The paper keeps this part in "high
+// precision"; it is not the path being optimised, so the kernel is a plain flash-style loop on the
+// legacy tensor-core MMA (mma.sync m16n8k16), correctness first:
+//   one CTA per (64 queries, head, batch), 4 warps of 16 query rows each; key/value tiles of 64
+//   rows staged in shared memory (V transposed, so both MMAs read 32-bit pairs); online softmax
+//   (running row maximum and sum, accumulators rescaled when the maximum moves); the probability
+//   fragment of the first MMA is reused as the A operand of the second.
+// Layout: q, k, v, o are [batch * seq, heads * 128] row-major with a common row stride `ld`
+// (elements), so the three inputs may also be column blocks of one fused buffer.
+#include "common.cuh"
+
+namespace bl {
+
+namespace {
+
+constexpr int kDh = 128;            // head dimension
+constexpr int kBq = 64;             // queries per CTA
+constexpr int kBk = 64;             // keys per tile
+constexpr int kKPad = kDh + 8;      // row pitch of the K tile (halves): 272 bytes, conflict-free 32-bit reads
+constexpr int kVPad = kBk + 8;      // row pitch of the transposed V tile
+
+__device__ __forceinline__ void mma_f16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
+  const __half2 h = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+__global__ void __launch_bounds__(128)
+attention_causal_kernel(const __half* __restrict__ q, const __half* __restrict__ k, const __half* __restrict__ v,
+                        __half* __restrict__ o, int S, int64_t ld, int64_t ld_o, float scale_log2) {
+  __shared__ __align__(16) __half Ks[kBk * kKPad];
+  __shared__ __align__(16) __half Vt[kDh * kVPad];
+  const int qb = blockIdx.x, head = blockIdx.y, batch = blockIdx.z;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, qd = lane & 3;
+  const int64_t tok0 = (int64_t)batch * S;
+  const __half* qh = q + tok0 * ld + (int64_t)head * kDh;
+  const __half* kh = k + tok0 * ld + (int64_t)head * kDh;
+  const __half* vh = v + tok0 * ld + (int64_t)head * kDh;
+  const int r0 = qb * kBq + warp * 16 + g, r1 = r0 + 8;          // the two query rows of this thread
+
+  // Q fragments of this warp's 16 rows, all 8 k-steps over d
+  uint32_t aq[8][4];
+#pragma unroll
+  for (int ks = 0; ks < 8; ++ks) {
+    const int d = ks * 16 + 2 * qd;
+    aq[ks][0] = *reinterpret_cast<const uint32_t*>(qh + (int64_t)r0 * ld + d);
+    aq[ks][1] = *reinterpret_cast<const uint32_t*>(qh + (int64_t)r1 * ld + d);
+    aq[ks][2] = *reinterpret_cast<const uint32_t*>(qh + (int64_t)r0 * ld + d + 8);
+    aq[ks][3] = *reinterpret_cast<const uint32_t*>(qh + (int64_t)r1 * ld + d + 8);
+  }
+  float acc[16][4];
+#pragma unroll
+  for (int dt = 0; dt < 16; ++dt) { acc[dt][0] = acc[dt][1] = acc[dt][2] = acc[dt][3] = 0.f; }
+  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+
+  for (int kb = 0; kb <= qb; ++kb) {
+    __syncthreads();                                             // previous tile fully consumed
+    // K tile: 64 keys x 128 d, 16 bytes per thread and step; V tile transposed on the way in
+    for (int idx = threadIdx.x; idx < kBk * (kDh / 8); idx += 128) {
+      const int key = idx / (kDh / 8), c = idx % (kDh / 8);
+      const int64_t row = (int64_t)(kb * kBk + key) * ld + c * 8;
+      *reinterpret_cast<uint4*>(&Ks[key * kKPad + c * 8]) = *reinterpret_cast<const uint4*>(kh + row);
+      const uint4 vv = *reinterpret_cast<const uint4*>(vh + row);
+      const __half* hv = reinterpret_cast<const __half*>(&vv);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) Vt[(c * 8 + j) * kVPad + key] = hv[j];
+    }
+    __syncthreads();
+
+    // S = Q K^T for this warp's 16 rows x 64 keys
+    float s[8][4];
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+      s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        const __half* kp = &Ks[(nt * 8 + g) * kKPad + ks * 16 + 2 * qd];
+        mma_f16(s[nt], aq[ks], *reinterpret_cast<const uint32_t*>(kp), *reinterpret_cast<const uint32_t*>(kp + 8));
+      }
+    }
+    if (kb == qb) {                                              // diagonal tile: keys after the query are masked
+#pragma unroll
+      for (int nt = 0; nt < 8; ++nt) {
+        const int key = kb * kBk + nt * 8 + 2 * qd;
+        if (key > r0) s[nt][0] = -INFINITY;
+        if (key + 1 > r0) s[nt][1] = -INFINITY;
+        if (key > r1) s[nt][2] = -INFINITY;
+        if (key + 1 > r1) s[nt][3] = -INFINITY;
+      }
+    }
+    // online softmax: new row maxima (over the 4 lanes that share a row), rescale, exponentials
+    float mx0 = m0, mx1 = m1;
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+      mx0 = fmaxf(mx0, fmaxf(s[nt][0], s[nt][1]));
+      mx1 = fmaxf(mx1, fmaxf(s[nt][2], s[nt][3]));
+    }
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 1)); mx0 = fmaxf(mx0, __shfl_xor_sync(0xFFFFFFFFu, mx0, 2));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xFFFFFFFFu, mx1, 2));
+    const float c0 = exp2f((m0 - mx0) * scale_log2), c1 = exp2f((m1 - mx1) * scale_log2);
+    m0 = mx0; m1 = mx1;
+    l0 *= c0; l1 *= c1;
+#pragma unroll
+    for (int dt = 0; dt < 16; ++dt) { acc[dt][0] *= c0; acc[dt][1] *= c0; acc[dt][2] *= c1; acc[dt][3] *= c1; }
+    uint32_t ap[4][4];                                           // P as A fragments: 4 k-steps of 16 keys
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+      const float p0 = exp2f((s[nt][0] - m0) * scale_log2), p1 = exp2f((s[nt][1] - m0) * scale_log2);
+      const float p2 = exp2f((s[nt][2] - m1) * scale_log2), p3 = exp2f((s[nt][3] - m1) * scale_log2);
+      l0 += p0 + p1; l1 += p2 + p3;
+      ap[nt >> 1][(nt & 1) * 2 + 0] = pack_half2(p0, p1);
+      ap[nt >> 1][(nt & 1) * 2 + 1] = pack_half2(p2, p3);
+    }
+    // O += P V
+#pragma unroll
+    for (int dt = 0; dt < 16; ++dt) {
+#pragma unroll
+      for (int kt = 0; kt < 4; ++kt) {
+        const __half* vp = &Vt[(dt * 8 + g) * kVPad + kt * 16 + 2 * qd];
+        mma_f16(acc[dt], ap[kt], *reinterpret_cast<const uint32_t*>(vp), *reinterpret_cast<const uint32_t*>(vp + 8));
+      }
+    }
+  }
+  // normalise and store
+  l0 += __shfl_xor_sync(0xFFFFFFFFu, l0, 1); l0 += __shfl_xor_sync(0xFFFFFFFFu, l0, 2);
+  l1 += __shfl_xor_sync(0xFFFFFFFFu, l1, 1); l1 += __shfl_xor_sync(0xFFFFFFFFu, l1, 2);
+  const float i0 = 1.f / l0, i1 = 1.f / l1;
+  __half* oh = o + tok0 * ld_o + (int64_t)head * kDh;
+#pragma unroll
+  for (int dt = 0; dt < 16; ++dt) {
+    const int d = dt * 8 + 2 * qd;
+    *reinterpret_cast<uint32_t*>(oh + (int64_t)r0 * ld_o + d) = pack_half2(acc[dt][0] * i0, acc[dt][1] * i0);
+    *reinterpret_cast<uint32_t*>(oh + (int64_t)r1 * ld_o + d) = pack_half2(acc[dt][2] * i1, acc[dt][3] * i1);
+  }
+}
+
+// y += r (residual), or y = max(y, 0): the block's elementwise glue, 8 halves per thread.
+__global__ void __launch_bounds__(256)
+add_inplace_kernel(__half* __restrict__ y, const __half* __restrict__ r, int64_t n8) {
+  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (i >= n8) return;
+  uint4 a = reinterpret_cast<uint4*>(y)[i];
+  const uint4 b = __ldg(reinterpret_cast<const uint4*>(r) + i);
+  __half2* pa = reinterpret_cast<__half2*>(&a);
+  const __half2* pb = reinterpret_cast<const __half2*>(&b);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) pa[j] = __hadd2(pa[j], pb[j]);
+  reinterpret_cast<uint4*>(y)[i] = a;
+}
+__global__ void __launch_bounds__(256)
+relu_inplace_kernel(__half* __restrict__ y, int64_t n8) {
+  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (i >= n8) return;
+  uint4 a = reinterpret_cast<uint4*>(y)[i];
+  __half2* pa = reinterpret_cast<__half2*>(&a);
+  const __half2 z = __float2half2_rn(0.f);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) pa[j] = __hmax2(pa[j], z);
+  reinterpret_cast<uint4*>(y)[i] = a;
+}
+
+}  // namespace
+
+cudaError_t launch_attention_causal(const void* q, const void* k, const void* v, void* o, int batch, int S,
+                                    int heads, int64_t ld, int64_t ld_o, cudaStream_t s) {
+  const float scale_log2 = 1.4426950408889634f / sqrtf((float)kDh);
+  dim3 grid((unsigned)(S / kBq), (unsigned)heads, (unsigned)batch);
+  attention_causal_kernel<<<grid, 128, 0, s>>>(reinterpret_cast<const __half*>(q), reinterpret_cast<const __half*>(k),
+                                               reinterpret_cast<const __half*>(v), reinterpret_cast<__half*>(o), S,
+                                               ld, ld_o, scale_log2);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_add_inplace(void* y, const void* r, int64_t n, cudaStream_t s) {
+  const int64_t n8 = n / 8;
+  add_inplace_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, s>>>(reinterpret_cast<__half*>(y),
+                                                                  reinterpret_cast<const __half*>(r), n8);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_relu_inplace(void* y, int64_t n, cudaStream_t s) {
+  const int64_t n8 = n / 8;
+  relu_inplace_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, s>>>(reinterpret_cast<__half*>(y), n8);
+  return cudaGetLastError();
+}
+
+}  // namespace bl

@@ -144,6 +144,12 @@ struct GemvArgs {
 };
 cudaError_t launch_gemv_decode(const GemvArgs& a, cudaStream_t s);
 
+// Decoder-block glue (fp16): causal attention core and the elementwise steps.
+cudaError_t launch_attention_causal(const void* q, const void* k, const void* v, void* o, int batch, int S,
+                                    int heads, int64_t ld, int64_t ld_o, cudaStream_t s);
+cudaError_t launch_add_inplace(void* y, const void* r, int64_t n, cudaStream_t s);   // y += r, n % 8 == 0
+cudaError_t launch_relu_inplace(void* y, int64_t n, cudaStream_t s);                 // y = max(y, 0)
+
 // Host-side layout maps (also exported through bitlinear_layout_index).
 int64_t prefill_bytes(int64_t N, int64_t K);
 void prefill_index(int64_t K, int64_t n, int64_t k, int64_t* byte_off, int* bit);

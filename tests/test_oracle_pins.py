@@ -384,3 +384,58 @@ def test_bad_shapes_are_rejected():
         O.binarize(np.zeros((2, 12), np.float32))            # K % 8 != 0
     with pytest.raises(ValueError):
         O.quant_act(np.zeros((2, 16), np.float32), G=4)      # K % (8 G) != 0
+
+
+# ---------------------------------------------------------------- attention core of the block (Sec. 2)
+
+def _attn_inputs(B, S, H, D, seed):
+    rng = np.random.default_rng(seed)
+    return [rng.standard_normal((B * S, H * D)).astype(np.float32) for _ in range(3)]
+
+
+def test_attention_matches_library_routine():
+    # special case that reduces to a library routine: torch's CPU scaled_dot_product_attention in fp64
+    import torch
+    B, S, H, D = 2, 80, 3, 16
+    q, k, v = _attn_inputs(B, S, H, D, 0)
+    out = O.attention_rows(q, k, v, B, S, H, D, np.arange(B * S))
+
+    def heads_first(a):
+        return torch.from_numpy(a).double().view(B, S, H, D).permute(0, 2, 1, 3)
+
+    ref = torch.nn.functional.scaled_dot_product_attention(heads_first(q), heads_first(k), heads_first(v), is_causal=True)
+    ref = ref.permute(0, 2, 1, 3).reshape(B * S, H * D).numpy()
+    assert np.abs(out - ref).max() < 1e-12
+
+
+def test_attention_closed_forms():
+    B, S, H, D = 2, 33, 2, 8
+    q, k, v = _attn_inputs(B, S, H, D, 1)
+    rows = np.arange(B * S)
+    out = O.attention_rows(q, k, v, B, S, H, D, rows)
+    # the first token of every sequence attends only itself
+    assert np.array_equal(out[0], v[0].astype(np.float64)) and np.array_equal(out[S], v[S].astype(np.float64))
+    # zero queries give uniform weights: the running mean of v over the causal prefix
+    out0 = O.attention_rows(np.zeros_like(q), k, v, B, S, H, D, rows)
+    for b in range(B):
+        prefix_mean = np.cumsum(v[b * S:(b + 1) * S].astype(np.float64), axis=0) / np.arange(1, S + 1)[:, None]
+        assert np.abs(out0[b * S:(b + 1) * S] - prefix_mean).max() < 1e-12
+    # outputs are convex combinations of the value rows seen so far, head by head
+    for t in (5, S + 7):
+        b, tt = divmod(t, S)
+        for h in range(H):
+            vs = v[b * S:b * S + tt + 1, h * D:(h + 1) * D]
+            assert (out[t, h * D:(h + 1) * D] <= vs.max(axis=0) + 1e-12).all()
+            assert (out[t, h * D:(h + 1) * D] >= vs.min(axis=0) - 1e-12).all()
+    # a future token never matters: changing k, v after position t leaves row t unchanged
+    k2, v2 = k.copy(), v.copy()
+    k2[20:S] += 3.0
+    v2[20:S] -= 2.0
+    out2 = O.attention_rows(q, k2, v2, B, S, H, D, np.arange(0, 20))
+    assert np.array_equal(out2, out[:20])
+    # a sharp query picks one key: q = c * k_s with large c selects v_s (s <= t)
+    q3 = np.zeros_like(q)
+    q3[10, :D] = 200.0 * k[4, :D] / (np.linalg.norm(k[4, :D]) ** 2) * np.sqrt(D) * 40
+    o3 = O.attention_rows(q3, k, v, B, S, H, D, np.array([10]))
+    scores = (q3[10, :D].astype(np.float64) @ k[:11, :D].astype(np.float64).T) / np.sqrt(D)
+    assert np.abs(o3[0, :D] - v[int(np.argmax(scores)), :D]).max() < 1e-6
