@@ -276,6 +276,8 @@ def run_b200(args):
             line["decode"] = bench_decode(B, synth, dev, peaks)
         if "pack" in parts:
             line["pack"] = bench_pack(B, synth, dev, peaks)
+        if "block" in parts:
+            line["block"] = bench_block(B, synth, dev, peaks)
         if "grouped" in parts:
             line["grouped"] = bench_grouped(B, synth, dev, peaks)
         if "cpu" in parts:
@@ -440,6 +442,44 @@ def bench_grouped(B, synth, dev, peaks):
             "forward_ms": t_fwd, "forward_tops": ops / t_fwd / 1e9}
 
 
+def bench_block(B, synth, dev, peaks):
+    """Config 4: one BitNet decoder block forward, d = 2048, 16 heads, FFN 8192, batch 4 x seq 2048,
+    fp16 activations, per-token quantisation; whole block and the attention core alone."""
+    batch, seq, heads, ffn = 4, 2048, 16, 8192
+    d, T = heads * 128, batch * seq
+    x = synth.make_x(T, d, torch.float16, seed=3, outliers=False).to(dev)
+    shapes = dict(q=(d, d), k=(d, d), v=(d, d), o=(d, d), up=(ffn, d), down=(d, ffn))
+    w = {n: B.binarize_pack(synth.make_w(N, K, torch.float32, seed=3 + 17 * i).to(dev), layout=B.PREFILL)
+         for i, (n, (N, K)) in enumerate(shapes.items())}
+    ws = torch.empty(B.workspace_bytes(B.OP_BLOCK_FORWARD, T, ffn, d, 1), dtype=torch.uint8, device=dev)
+    out = B.block_forward(x, w, batch, seq, heads, ffn, ws=ws)
+
+    def timed(fn, reps):
+        for _ in range(2):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    t_block = timed(lambda: B.block_forward(x, w, batch, seq, heads, ffn, ws=ws), 10)
+    t_attn = timed(lambda: B.attention_causal(out["q"], out["k"], out["v"], batch, seq, heads, o=out["a"]), 10)
+    assert B.ws_status(ws) == B.OK
+    lin_ops = 2.0 * T * (4 * d * d + 2 * d * ffn)
+    attn_flops = 4.0 * batch * heads * (seq * (seq + 1) / 2) * 128
+    return {"workload": "BitNet decoder block forward: d 2048, 16 heads, FFN 8192 (ReLU, eta form on the down "
+                        "input), batch 4 x seq 2048, fp16 activations, per-token quantisation, six BitLinear "
+                        "layers + causal fp16 attention + residuals",
+            "block_ms": t_block, "attention_ms": t_attn, "bitlinear_ops": lin_ops,
+            "bitlinear_tops_of_block_time": lin_ops / t_block / 1e9,
+            "attention_tflops": attn_flops / t_attn / 1e9,
+            "gpu_launches": 10 * 17}
+
+
 # --------------------------------------------------------------------------- the CPU oracle, timed
 
 def oracle_prefill_sample(x_host, W_host, tokens, reps=1):
@@ -524,8 +564,8 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
-    ap.add_argument("--parts", default="decode,pack,grouped,cpu",
-                    help="extra measurements beside the prefill step (comma list of decode, pack, grouped, cpu; "
+    ap.add_argument("--parts", default="decode,pack,grouped,block,cpu",
+                    help="extra measurements beside the prefill step (comma list of decode, pack, grouped, block, cpu; "
                          "'none' for the prefill step alone, e.g. under a profiler)")
     args = ap.parse_args()
     if args.impl == "reference":
