@@ -127,9 +127,9 @@ bl_status bitlinear_quant_act(const void* x, bl_dtype xt, int64_t M, int64_t K, 
  * given.  Such callers still own x, x_q, gamma and eta, but have nowhere to put the statistics
  * that the per-tensor path keeps between its two passes.
  *
- * The statistics go to a fixed array inside the library instead (about
- * 24 * BL_NOALLOC_MAX_SEGMENTS bytes, resident on every GPU that loads the library until the
- * process ends).  Consequences:
+ * The statistics go to a fixed array inside the library instead (24 bytes per segment for
+ * BL_NOALLOC_MAX_SEGMENTS segments plus a 0.26 MB header, about 0.7 MB in all, resident on every
+ * GPU that loads the library until the process ends).  Consequences:
  *   - BL_PER_TENSOR calls with M * G > BL_NOALLOC_MAX_SEGMENTS return BL_ERR_TOO_LARGE and launch
  *     nothing.  BL_PER_TOKEN calls need no scratch and have no such limit.
  *   - All calls on one GPU share the array.  Calls that may overlap on the GPU (different

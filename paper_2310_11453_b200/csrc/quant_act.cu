@@ -23,13 +23,20 @@ constexpr int kQuantThreads = 256;
 
 struct SegRecord {                 // per-segment record kept between the two per-tensor kernels
   double mean, rstd;
-  float xabs, pad;
+  float xlo, xhi;                  // raw extremes of the segment
 };
 
-struct TensorScope {               // workspace header for the per-tensor path
+struct TensorScope {               // running extremes of x^ per group (long-segment kernels, atomics)
   unsigned long long enc_min[BL_MAX_GROUPS];
   unsigned long long enc_max[BL_MAX_GROUPS];
 };
+struct ScopePartial {              // one CTA's extremes of x^ for one group (fast path, plain stores)
+  unsigned long long lo, hi;
+};
+constexpr int kMaxStatCtas = 256;  // upper bound on the grid of the persistent fast-path kernels
+// Per-tensor workspace: TensorScope | ScopePartial[kMaxStatCtas][BL_MAX_GROUPS] | SegRecord[M*G].
+constexpr size_t kWsHeaderBytes =
+    sizeof(TensorScope) + (size_t)kMaxStatCtas * BL_MAX_GROUPS * sizeof(ScopePartial);
 
 template <typename T>
 __device__ __forceinline__ void stage_segment(const T* __restrict__ src, int Kg, float* seg) {
@@ -90,7 +97,7 @@ tensor_stats(const T* __restrict__ x, int64_t K, int G, float ln_eps, TensorScop
   SegMoments mom; float xlo, xhi;
   segment_moments<kQuantThreads>(seg, Kg, ln_eps, red, mom, xlo, xhi);
   if (threadIdx.x == 0) {
-    recs[blockIdx.x] = SegRecord{mom.mean, mom.rstd, fmaxf(fabsf(xlo), fabsf(xhi)), 0.f};
+    recs[blockIdx.x] = SegRecord{mom.mean, mom.rstd, xlo, xhi};
     atomicMin(&sc->enc_min[g], enc_ordered64(((double)xlo - mom.mean) * mom.rstd));
     atomicMax(&sc->enc_max[g], enc_ordered64(((double)xhi - mom.mean) * mom.rstd));
   }
@@ -109,7 +116,7 @@ tensor_codes(const T* __restrict__ x, int64_t K, int G, int mode, const TensorSc
   const double lo = dec_ordered64(sc->enc_min[g]), hi = dec_ordered64(sc->enc_max[g]);
   double gam, et;
   scope_gamma_eta(mode, lo, hi, gam, et);
-  const QuantMap map = make_quant_map(mode, SegMoments{rec.mean, rec.rstd}, gam, et, rec.xabs);
+  const QuantMap map = make_quant_map(mode, SegMoments{rec.mean, rec.rstd}, gam, et, fmaxf(fabsf(rec.xlo), fabsf(rec.xhi)));
   if (m == 0 && threadIdx.x == 0) {
     gamma[g] = (float)gam;
     if (eta) eta[g] = (float)et;
@@ -125,24 +132,29 @@ tensor_codes(const T* __restrict__ x, int64_t K, int G, int mode, const TensorSc
 
 
 // ================================================================================================
-// Fast path: one warp per (token, group) segment, the whole segment held in registers.
+// Fast path: one warp per (token, group) segment, the segment staged in shared memory.
 //
-// Used when a segment fits 16 x 16 bytes per lane (K_g <= 4096 for 16-bit inputs, <= 2048 for
-// fp32), which covers every shape of the paper's model table.  A warp issues all loads of its
-// segment at once (up to 8 KB in flight per warp, 16 warps per SM), then takes the two LN passes
-// and the quantisation out of registers with warp shuffles only: no shared memory, no block
-// barrier.  Sums are fp32 inside a lane and fp64 across lanes; the second pass sums squared
-// deviations from the fp32-rounded mean and corrects for that rounding exactly.  Reciprocals and
-// the inverse square root are hardware seeds refined by Newton steps in fp64 (below one ulp of
-// fp64 after two steps), which keeps fp64 division and square-root routines out of the kernels.
-constexpr int kRowWarps = 8;
-constexpr int kRowRegs = 16;                                  // uint4 per lane
+// Used when a segment is a whole number of 256-element pieces and at most 8 KB (K_g <= 4096 for
+// 16-bit inputs, <= 2048 for fp32), which covers every shape of the paper's model table.  The
+// kernels are persistent: one CTA per SM; CTA c owns the contiguous segment range
+// [c*S/grid, (c+1)*S/grid) and its warps draw segments from it through a shared counter.  Each warp
+// has two 8 KB slots of shared memory: while it works on one, the asynchronous copies (cp.async,
+// 16 bytes per lane and instruction) of its next segment land in the other, so every warp keeps a
+// segment's worth of HBM traffic outstanding whatever it is computing.  Waiting is
+// cp.async.wait_group: no barrier objects, no spin loops.  A warp walks its segment in chunks of
+// 8 elements per lane (a short rolled loop: small code, few registers), with warp shuffles for
+// the reductions and no block barrier inside the loop.  Sums are fp32 inside a lane and fp64
+// across lanes, in one pass over deviations from a pilot value.  Reciprocals and the inverse
+// square root are hardware seeds refined by Newton steps in fp64 (below one ulp of fp64 after two
+// steps), which keeps fp64 division and square-root routines out of the kernels.
+constexpr int kRowWarps = 12;
+constexpr int kSlotBytes = 8192;
+constexpr int kRowStage = kRowWarps * 2 * kSlotBytes;
 constexpr float kRoundMagic = 12582912.f;                     // 1.5 * 2^23: x + magic - magic = rne(x), |x| < 2^22
 
 template <typename T> struct RowTraits {                      // chunk = 8 consecutive elements
-  static constexpr int kVecPerChunk = sizeof(T) == 4 ? 2 : 1;
-  static constexpr int kChunks = kRowRegs / kVecPerChunk;     // chunks per lane
-  static constexpr int kMaxKg = kChunks * 32 * 8;
+  static constexpr int kVecPerChunk = sizeof(T) == 4 ? 2 : 1; // 16-byte pieces per chunk
+  static constexpr int kMaxKg = kSlotBytes / (int)sizeof(T);
 };
 
 __device__ __forceinline__ double rcp_newton(double d) {      // d > 0
@@ -158,104 +170,89 @@ __device__ __forceinline__ double rsqrt_newton(double d) {    // d >= 0
   return y * (1.5 - 0.5 * d * y * y);
 }
 
-template <typename T>
-__device__ __forceinline__ void row_load(const T* __restrict__ src, int nchunks, int lane, uint4 (&raw)[kRowRegs]) {
-  constexpr int V = RowTraits<T>::kVecPerChunk;
-#pragma unroll
-  for (int i = 0; i < RowTraits<T>::kChunks; ++i) {
-    const int c = lane + 32 * i;
-#pragma unroll
-    for (int j = 0; j < V; ++j) {
-      raw[i * V + j] = make_uint4(0u, 0u, 0u, 0u);
-      if (c < nchunks) raw[i * V + j] = __ldg(reinterpret_cast<const uint4*>(src + (size_t)c * 8) + j);
-    }
-  }
-}
-
-template <typename T> __device__ __forceinline__ void row_unpack(const uint4 (&raw)[kRowRegs], int i, float (&v)[8]);
-template <> __device__ __forceinline__ void row_unpack<float>(const uint4 (&raw)[kRowRegs], int i, float (&v)[8]) {
-  const uint4 a = raw[2 * i], b = raw[2 * i + 1];
-  v[0] = __uint_as_float(a.x); v[1] = __uint_as_float(a.y); v[2] = __uint_as_float(a.z); v[3] = __uint_as_float(a.w);
-  v[4] = __uint_as_float(b.x); v[5] = __uint_as_float(b.y); v[6] = __uint_as_float(b.z); v[7] = __uint_as_float(b.w);
-}
-template <> __device__ __forceinline__ void row_unpack<__half>(const uint4 (&raw)[kRowRegs], int i, float (&v)[8]) {
-  const uint32_t w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[j]));
-    v[2 * j] = f.x; v[2 * j + 1] = f.y;
-  }
-}
-template <> __device__ __forceinline__ void row_unpack<__nv_bfloat16>(const uint4 (&raw)[kRowRegs], int i, float (&v)[8]) {
-  const uint32_t w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    v[2 * j] = __uint_as_float(w[j] << 16);
-    v[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
-  }
-}
-
-struct RowStats { double mean, rstd; float xlo, xhi; };
-
 template <typename H2> __device__ __forceinline__ H2 as_h2(uint32_t w) { return *reinterpret_cast<H2*>(&w); }
 template <typename H2> __device__ __forceinline__ uint32_t h2_bits(H2 h) { return *reinterpret_cast<uint32_t*>(&h); }
 
-// Eq. 12 statistics of the segment held in raw[]: every lane returns the same values.
+// Chunk c of a staged segment (8 consecutive elements) as fp32.
+template <typename T> struct Chunk;
+template <> struct Chunk<float> {
+  uint4 a, b;
+  __device__ __forceinline__ void load(const uint4* slot, int c) { a = slot[2 * c]; b = slot[2 * c + 1]; }
+  __device__ __forceinline__ void unpack(float (&v)[8]) const {
+    v[0] = __uint_as_float(a.x); v[1] = __uint_as_float(a.y); v[2] = __uint_as_float(a.z); v[3] = __uint_as_float(a.w);
+    v[4] = __uint_as_float(b.x); v[5] = __uint_as_float(b.y); v[6] = __uint_as_float(b.z); v[7] = __uint_as_float(b.w);
+  }
+};
+template <> struct Chunk<__half> {
+  uint4 a;
+  __device__ __forceinline__ void load(const uint4* slot, int c) { a = slot[c]; }
+  __device__ __forceinline__ void unpack(float (&v)[8]) const {
+    const uint32_t w[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float2 f = __half22float2(as_h2<__half2>(w[j]));
+      v[2 * j] = f.x; v[2 * j + 1] = f.y;
+    }
+  }
+};
+template <> struct Chunk<__nv_bfloat16> {
+  uint4 a;
+  __device__ __forceinline__ void load(const uint4* slot, int c) { a = slot[c]; }
+  __device__ __forceinline__ void unpack(float (&v)[8]) const {
+    const uint32_t w[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      v[2 * j] = __uint_as_float(w[j] << 16);
+      v[2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+    }
+  }
+};
+
+struct RowStats { double mean, rstd; float xlo, xhi; };
+
+// Eq. 12 statistics of the staged segment (ni chunks per lane): every lane returns the same values.
 // One pass: deviations are taken from a pilot value c (the mean of the segment's first 8
 // elements), which keeps sum (x - c) and sum (x - c)^2 small and well conditioned:
 //   mean = c + sum (x - c) / K,   Var = sum (x - c)^2 / K - (mean - c)^2.
 template <typename T>
-__device__ __forceinline__ RowStats row_stats(const uint4 (&raw)[kRowRegs], int nchunks, int lane, float ln_eps,
-                                              double inv_kg) {
-  float pilot = 0.f;
+__device__ __forceinline__ RowStats row_stats(const uint4* slot, int ni, int lane, float ln_eps, double inv_kg) {
+  float pilot;
   {
-    float v[8];
-    row_unpack<T>(raw, 0, v);                        // lane 0 holds chunk 0
+    Chunk<T> ch; float v[8];
+    ch.load(slot, 0); ch.unpack(v);                  // same address in every lane: a broadcast
     pilot = 0.125f * (((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7])));
-    pilot = __shfl_sync(0xFFFFFFFFu, pilot, 0);
     if (ln_eps < 0.f) pilot = 0.f;
   }
   float s = 0.f, q = 0.f, mn = INFINITY, mx = -INFINITY;
-  uint32_t plo = 0, phi = 0;
-  bool have16 = false;
+  uint32_t plo = slot[0].x, phi = plo;               // 16-bit inputs: running packed extremes
+#pragma unroll 4
+  for (int i = 0; i < ni; ++i) {
+    Chunk<T> ch; float v[8], d[8];
+    ch.load(slot, lane + 32 * i); ch.unpack(v);
 #pragma unroll
-  for (int i = 0; i < RowTraits<T>::kChunks; ++i) {
-    if (lane + 32 * i < nchunks) {
-      float v[8];
-      row_unpack<T>(raw, i, v);
-      float d[8];
+    for (int j = 0; j < 8; ++j) d[j] = v[j] - pilot;
+    s += ((d[0] + d[1]) + (d[2] + d[3])) + ((d[4] + d[5]) + (d[6] + d[7]));
+    float p0 = d[0] * d[0], p1 = d[1] * d[1];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) d[j] = v[j] - pilot;
-      s += ((d[0] + d[1]) + (d[2] + d[3])) + ((d[4] + d[5]) + (d[6] + d[7]));
-      float p = 0.f;
+    for (int j = 2; j < 8; j += 2) { p0 = fmaf(d[j], d[j], p0); p1 = fmaf(d[j + 1], d[j + 1], p1); }
+    q += p0 + p1;
+    if constexpr (sizeof(T) == 4) {
 #pragma unroll
-      for (int j = 0; j < 8; ++j) p = fmaf(d[j], d[j], p);
-      q += p;
-      if constexpr (sizeof(T) == 4) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) { mn = fminf(mn, v[j]); mx = fmaxf(mx, v[j]); }
-      } else {
-        using H2 = typename std::conditional<std::is_same<T, __half>::value, __half2, __nv_bfloat162>::type;
-        const uint32_t w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
-        H2 a = __hmin2(__hmin2(as_h2<H2>(w[0]), as_h2<H2>(w[1])), __hmin2(as_h2<H2>(w[2]), as_h2<H2>(w[3])));
-        H2 b = __hmax2(__hmax2(as_h2<H2>(w[0]), as_h2<H2>(w[1])), __hmax2(as_h2<H2>(w[2]), as_h2<H2>(w[3])));
-        if (have16) { a = __hmin2(a, as_h2<H2>(plo)); b = __hmax2(b, as_h2<H2>(phi)); }
-        plo = h2_bits(a); phi = h2_bits(b); have16 = true;
-      }
+      for (int j = 0; j < 8; ++j) { mn = fminf(mn, v[j]); mx = fmaxf(mx, v[j]); }
+    } else {
+      using H2 = typename std::conditional<std::is_same<T, __half>::value, __half2, __nv_bfloat162>::type;
+      const uint32_t w[4] = {ch.a.x, ch.a.y, ch.a.z, ch.a.w};
+      const H2 a = __hmin2(__hmin2(as_h2<H2>(w[0]), as_h2<H2>(w[1])), __hmin2(as_h2<H2>(w[2]), as_h2<H2>(w[3])));
+      const H2 b = __hmax2(__hmax2(as_h2<H2>(w[0]), as_h2<H2>(w[1])), __hmax2(as_h2<H2>(w[2]), as_h2<H2>(w[3])));
+      plo = h2_bits(__hmin2(a, as_h2<H2>(plo))); phi = h2_bits(__hmax2(b, as_h2<H2>(phi)));
     }
   }
-  if constexpr (sizeof(T) != 4) {
-    if (have16) {
-      using H2 = typename std::conditional<std::is_same<T, __half>::value, __half2, __nv_bfloat162>::type;
-      const H2 a = as_h2<H2>(plo), b = as_h2<H2>(phi);
-      if constexpr (std::is_same<T, __half>::value) {
-        const float2 fa = __half22float2(a), fb = __half22float2(b);
-        mn = fminf(fa.x, fa.y); mx = fmaxf(fb.x, fb.y);
-      } else {
-        const float2 fa = __bfloat1622float2(a), fb = __bfloat1622float2(b);
-        mn = fminf(fa.x, fa.y); mx = fmaxf(fb.x, fb.y);
-      }
-    }
+  if constexpr (std::is_same<T, __half>::value) {
+    const float2 fa = __half22float2(as_h2<__half2>(plo)), fb = __half22float2(as_h2<__half2>(phi));
+    mn = fminf(fa.x, fa.y); mx = fmaxf(fb.x, fb.y);
+  } else if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+    const float2 fa = __bfloat1622float2(as_h2<__nv_bfloat162>(plo)), fb = __bfloat1622float2(as_h2<__nv_bfloat162>(phi));
+    mn = fminf(fa.x, fa.y); mx = fmaxf(fb.x, fb.y);
   }
   const double S = warp_sum((double)s), Q = warp_sum((double)q);
   RowStats st;
@@ -273,130 +270,285 @@ struct RowMap {            // Quant of Eq. 4-6 as one fp32 FMA, plus what the ex
   double mean, rstd, eta, scale;
   float A, B, tau;
   int code_lo;
+  bool clip;               // some element of the segment may reach a clip bound (uniform over the segment)
 };
-__device__ __forceinline__ RowMap row_map(int mode, double mean, double rstd, double gamma, double eta, float xabs) {
+__device__ __forceinline__ RowMap row_map(int mode, double mean, double rstd, double gamma, double eta, float xlo,
+                                          float xhi) {
   RowMap m;
   m.mean = mean; m.rstd = rstd; m.eta = eta;
   m.scale = gamma > 0.0 ? (double)kQb * rcp_newton(gamma) : 0.0;
   m.A = (float)(rstd * m.scale);
   m.B = (float)(-(mean * rstd + eta) * m.scale);
-  m.tau = 4e-7f * (fabsf(m.A) * xabs + fabsf(m.B) + 1.0f);
+  m.tau = 4e-7f * (fabsf(m.A) * fmaxf(fabsf(xlo), fabsf(xhi)) + fabsf(m.B) + 1.0f);
   m.code_lo = (mode == BL_ABSMAX) ? -kCodeMax : 0;
+  // A >= 0, so x*A + B over the segment spans [xlo*A + B, xhi*A + B]: a quarter inside the
+  // bounds, rounding cannot leave them and the clip of Eq. 4 / 6 is the identity.
+  m.clip = !(fmaf(xlo, m.A, m.B) > (float)m.code_lo - 0.25f && fmaf(xhi, m.A, m.B) < (float)kCodeMax + 0.25f);
   return m;
 }
-// The rare element too close to a rounding tie for fp32: the equations in fp64, in their order.
-__device__ __noinline__ int row_code_exact(float x, double mean, double rstd, double eta, double scale) {
+// The rare chunk with an element too close to a rounding tie for fp32: the equations in fp64,
+// in their order, four elements per call.
+__device__ __forceinline__ uint32_t row_code_exact(float x, double mean, double rstd, double eta, double scale,
+                                                   int code_lo) {
   const double xh = ((double)x - mean) * rstd;
-  return (int)rint((xh - eta) * scale);
+  return (uint32_t)(max(code_lo, min(kCodeMax, (int)rint((xh - eta) * scale))) & 0xFF);
 }
+__device__ __noinline__ uint32_t row_codes4_exact(float v0, float v1, float v2, float v3, double mean, double rstd,
+                                                  double eta, double scale, int code_lo) {
+  return row_code_exact(v0, mean, rstd, eta, scale, code_lo) | row_code_exact(v1, mean, rstd, eta, scale, code_lo) << 8 |
+         row_code_exact(v2, mean, rstd, eta, scale, code_lo) << 16 |
+         row_code_exact(v3, mean, rstd, eta, scale, code_lo) << 24;
+}
+template <bool kClip>
 __device__ __forceinline__ uint2 row_codes8(const float (&v)[8], const RowMap& m) {
-  // f is clipped in fp32 (the clip bounds are integers, so clip and rne commute); adding the
-  // magic constant leaves rne(f) as a two's-complement byte in the low bits of the sum.
+  // Adding the magic constant leaves rne(f) as a two's-complement byte in the low bits of the
+  // sum.  With kClip, f is clipped in fp32 first (the bounds are integers, so clip and rne
+  // commute).  dist collects max |f - rne(f)| to spot elements within tau of a rounding tie
+  // (and, with kClip, elements the clip moved: both go to the exact redo).
   uint32_t t[8];
-  bool near_tie = false;
-  const float lo = (float)m.code_lo, hi = (float)kCodeMax, edge = 0.5f - m.tau;
+  float dist = 0.f;
+  const float lo = (float)m.code_lo, hi = (float)kCodeMax;
 #pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const float f = fmaf(v[j], m.A, m.B);
-    const float tj = fminf(fmaxf(f, lo), hi) + kRoundMagic;
-    near_tie |= fabsf(f - (tj - kRoundMagic)) > edge;         // inside the clip range: within tau of a tie
-    t[j] = __float_as_uint(tj);
+  for (int j = 0; j < 8; j += 2) {
+    const float f0 = fmaf(v[j], m.A, m.B), f1 = fmaf(v[j + 1], m.A, m.B);
+    const float t0 = (kClip ? fminf(fmaxf(f0, lo), hi) : f0) + kRoundMagic;
+    const float t1 = (kClip ? fminf(fmaxf(f1, lo), hi) : f1) + kRoundMagic;
+    dist = fmaxf(fmaxf(dist, fabsf(f0 - (t0 - kRoundMagic))), fabsf(f1 - (t1 - kRoundMagic)));
+    t[j] = __float_as_uint(t0); t[j + 1] = __float_as_uint(t1);
   }
   uint2 out;
   out.x = __byte_perm(__byte_perm(t[0], t[1], 0x0040), __byte_perm(t[2], t[3], 0x0040), 0x5410);
   out.y = __byte_perm(__byte_perm(t[4], t[5], 0x0040), __byte_perm(t[6], t[7], 0x0040), 0x5410);
-  if (near_tie) {                                            // rare: redo the 8 codes exactly
-    uint32_t w[2] = {0u, 0u};
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int c = max(m.code_lo, min(kCodeMax, row_code_exact(v[j], m.mean, m.rstd, m.eta, m.scale)));
-      w[j >> 2] |= (uint32_t)(c & 0xFF) << (8 * (j & 3));
-    }
-    out = make_uint2(w[0], w[1]);
+  if (dist > 0.5f - m.tau) {                                 // rare
+    out.x = row_codes4_exact(v[0], v[1], v[2], v[3], m.mean, m.rstd, m.eta, m.scale, m.code_lo);
+    out.y = row_codes4_exact(v[4], v[5], v[6], v[7], m.mean, m.rstd, m.eta, m.scale, m.code_lo);
   }
   return out;
 }
 
-template <typename T>
-__device__ __forceinline__ void row_store_codes(const uint4 (&raw)[kRowRegs], int nchunks, int lane, const RowMap& map,
-                                                int8_t* __restrict__ dst) {
-#pragma unroll
-  for (int i = 0; i < RowTraits<T>::kChunks; ++i) {
+template <typename T, bool kClip>
+__device__ __forceinline__ void row_store_codes_impl(const uint4* slot, int ni, int lane, const RowMap& map,
+                                                     int8_t* __restrict__ dst) {
+#pragma unroll 2
+  for (int i = 0; i < ni; ++i) {
     const int c = lane + 32 * i;
-    if (c < nchunks) {
-      float v[8];
-      row_unpack<T>(raw, i, v);
-      *reinterpret_cast<uint2*>(dst + (size_t)c * 8) = row_codes8(v, map);
-    }
+    Chunk<T> ch; float v[8];
+    ch.load(slot, c); ch.unpack(v);
+    *reinterpret_cast<uint2*>(dst + (size_t)c * 8) = row_codes8<kClip>(v, map);
   }
+}
+template <typename T>
+__device__ __forceinline__ void row_store_codes(const uint4* slot, int ni, int lane, const RowMap& map,
+                                                int8_t* __restrict__ dst) {
+  if (map.clip) row_store_codes_impl<T, true>(slot, ni, lane, map, dst);
+  else row_store_codes_impl<T, false>(slot, ni, lane, map, dst);
+}
+
+// ---- segment ranges and staging --------------------------------------------------------------------
+struct RowRange { int64_t begin, end; };
+__device__ __forceinline__ RowRange cta_range(int64_t segments) {
+  RowRange r;
+  r.begin = segments * (int64_t)blockIdx.x / (int64_t)gridDim.x;
+  r.end = segments * ((int64_t)blockIdx.x + 1) / (int64_t)gridDim.x;
+  return r;
+}
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
+               "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+// All of this thread's copy groups but the newest are complete; __syncwarp() makes the other
+// lanes' pieces visible too.
+__device__ __forceinline__ void cp_async_wait_but_newest() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
+
+// Draws the warp's next segment (-1 when the CTA's range is used up), starts its copy into
+// `slot` and closes the copy group (an empty one when there is nothing left to copy).
+// reverse walks the range from its end: the second per-tensor pass then begins with the rows the
+// first pass read last, the ones most likely still in L2.
+template <typename T>
+__device__ __forceinline__ int64_t stage_next(const T* __restrict__ x, const RowRange& rg, int64_t K, int G, int Kg,
+                                              bool reverse, int* counter, uint4* slot, int lane) {
+  int r = 0;
+  if (lane == 0) r = atomicAdd(counter, 1);
+  r = __shfl_sync(0xFFFFFFFFu, r, 0);
+  int64_t seg = -1;
+  if (rg.begin + r < rg.end) {
+    seg = reverse ? rg.end - 1 - r : rg.begin + r;
+    const uint4* src = reinterpret_cast<const uint4*>(x + (seg / G) * K + (seg % G) * (int64_t)Kg);
+    const int nv = Kg / 256 * RowTraits<T>::kVecPerChunk;      // 16-byte pieces per lane
+#pragma unroll 4
+    for (int i = 0; i < nv; ++i) cp_async16(slot + lane + 32 * i, src + lane + 32 * i);
+  }
+  cp_async_commit();
+  return seg;
+}
+
+// The warp loop shared by the three kernels: body(seg, slot) runs with the segment staged and
+// the next one already on its way.
+template <typename T, typename Body>
+__device__ __forceinline__ void for_each_segment(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg,
+                                                 bool reverse, int* counter, unsigned char* stage, int64_t first_seg,
+                                                 Body body) {
+  const int lane = threadIdx.x & 31;
+  uint4* slots = reinterpret_cast<uint4*>(stage + (size_t)(threadIdx.x >> 5) * 2 * kSlotBytes);
+  const RowRange rg = cta_range(segments);
+  int cur = 0;
+  int64_t seg = first_seg;
+  while (seg >= 0) {
+    const int64_t next = stage_next<T>(x, rg, K, G, Kg, reverse, counter, slots + (cur ^ 1) * (kSlotBytes / 16), lane);
+    cp_async_wait_but_newest();
+    __syncwarp();
+    body(seg, slots + cur * (kSlotBytes / 16));
+    __syncwarp();                                    // every lane is done with the slot before it is refilled
+    seg = next; cur ^= 1;
+  }
+}
+// First draw of a warp (into slot 0), split off so that a kernel can put work between it and the loop.
+template <typename T>
+__device__ __forceinline__ int64_t first_segment(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg,
+                                                 bool reverse, int* counter, unsigned char* stage) {
+  uint4* slots = reinterpret_cast<uint4*>(stage + (size_t)(threadIdx.x >> 5) * 2 * kSlotBytes);
+  return stage_next<T>(x, cta_range(segments), K, G, Kg, reverse, counter, slots, threadIdx.x & 31);
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kRowWarps * 32, 2)
+__global__ void __launch_bounds__(kRowWarps * 32, 1)
 rows_per_token(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg, int mode, float ln_eps,
                double inv_kg, int8_t* __restrict__ x_q, float* __restrict__ gamma, float* __restrict__ eta) {
+  extern __shared__ __align__(16) unsigned char stage[];
+  __shared__ int counter;
   const int lane = threadIdx.x & 31;
-  const int64_t seg = (int64_t)blockIdx.x * kRowWarps + (threadIdx.x >> 5);
-  if (seg >= segments) return;                                   // whole warp
-  const int64_t base = (seg / G) * K + (seg % G) * (int64_t)Kg;
-  const int nchunks = Kg / 8;
-  uint4 raw[kRowRegs];
-  row_load<T>(x + base, nchunks, lane, raw);
-  const RowStats st = row_stats<T>(raw, nchunks, lane, ln_eps, inv_kg);
-  const double lo = ((double)st.xlo - st.mean) * st.rstd, hi = ((double)st.xhi - st.mean) * st.rstd;
-  double gam, et;
-  scope_gamma_eta(mode, lo, hi, gam, et);
-  const RowMap map = row_map(mode, st.mean, st.rstd, gam, et, fmaxf(fabsf(st.xlo), fabsf(st.xhi)));
-  if (lane == 0) {
-    gamma[seg] = (float)gam;
-    if (eta) eta[seg] = (float)et;
-  }
-  row_store_codes<T>(raw, nchunks, lane, map, x_q + base);
+  if (threadIdx.x == 0) counter = 0;
+  __syncthreads();
+  const int ni = Kg / 256;
+  const int64_t first = first_segment<T>(x, segments, K, G, Kg, false, &counter, stage);
+  for_each_segment<T>(x, segments, K, G, Kg, false, &counter, stage, first, [&](int64_t seg, const uint4* slot) {
+    const RowStats st = row_stats<T>(slot, ni, lane, ln_eps, inv_kg);
+    const double lo = ((double)st.xlo - st.mean) * st.rstd, hi = ((double)st.xhi - st.mean) * st.rstd;
+    double gam, et;
+    scope_gamma_eta(mode, lo, hi, gam, et);
+    const RowMap map = row_map(mode, st.mean, st.rstd, gam, et, st.xlo, st.xhi);
+    if (lane == 0) {
+      gamma[seg] = (float)gam;
+      if (eta) eta[seg] = (float)et;
+    }
+    row_store_codes<T>(slot, ni, lane, map, x_q + (seg / G) * K + (seg % G) * (int64_t)Kg);
+  });
 }
 
+// Per-tensor scope, first pass: the segment records, and per CTA and group the extremes of x^ on
+// the order-preserving encoding (plain stores: every CTA writes its own G entries, the second pass
+// folds them; no atomics on global memory and nothing to initialise).
 template <typename T>
-__global__ void __launch_bounds__(kRowWarps * 32, 3)
+__global__ void __launch_bounds__(kRowWarps * 32, 1)
 rows_tensor_stats(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg, float ln_eps, double inv_kg,
-                  TensorScope* sc, SegRecord* __restrict__ recs) {
+                  ScopePartial* __restrict__ partials, SegRecord* __restrict__ recs) {
+  extern __shared__ __align__(16) unsigned char stage[];
+  __shared__ int counter;
+  __shared__ unsigned long long part_lo[BL_MAX_GROUPS], part_hi[BL_MAX_GROUPS];
   const int lane = threadIdx.x & 31;
-  const int64_t seg = (int64_t)blockIdx.x * kRowWarps + (threadIdx.x >> 5);
-  if (seg >= segments) return;
-  const int g = (int)(seg % G);
-  const int64_t base = (seg / G) * K + g * (int64_t)Kg;
-  const int nchunks = Kg / 8;
-  uint4 raw[kRowRegs];
-  row_load<T>(x + base, nchunks, lane, raw);
-  const RowStats st = row_stats<T>(raw, nchunks, lane, ln_eps, inv_kg);
-  if (lane == 0) {
-    recs[seg] = SegRecord{st.mean, st.rstd, fmaxf(fabsf(st.xlo), fabsf(st.xhi)), 0.f};
-    atomicMin(&sc->enc_min[g], enc_ordered64(((double)st.xlo - st.mean) * st.rstd));
-    atomicMax(&sc->enc_max[g], enc_ordered64(((double)st.xhi - st.mean) * st.rstd));
+  if (threadIdx.x == 0) counter = 0;
+  if (threadIdx.x < BL_MAX_GROUPS) { part_lo[threadIdx.x] = ~0ull; part_hi[threadIdx.x] = 0ull; }
+  __syncthreads();
+  const int ni = Kg / 256;
+  const int64_t first = first_segment<T>(x, segments, K, G, Kg, false, &counter, stage);
+  for_each_segment<T>(x, segments, K, G, Kg, false, &counter, stage, first, [&](int64_t seg, const uint4* slot) {
+    const RowStats st = row_stats<T>(slot, ni, lane, ln_eps, inv_kg);
+    if (lane == 0) {
+      const int g = (int)(seg % G);
+      recs[seg] = SegRecord{st.mean, st.rstd, st.xlo, st.xhi};
+      atomicMin(&part_lo[g], enc_ordered64(((double)st.xlo - st.mean) * st.rstd));
+      atomicMax(&part_hi[g], enc_ordered64(((double)st.xhi - st.mean) * st.rstd));
+    }
+  });
+  __syncthreads();
+  if (threadIdx.x < G)
+    partials[(size_t)blockIdx.x * G + threadIdx.x] = ScopePartial{part_lo[threadIdx.x], part_hi[threadIdx.x]};
+}
+
+// Second pass: folds the first pass's `stat_ctas` partial extremes into gamma / eta per group,
+// then writes the codes.
+template <typename T>
+__global__ void __launch_bounds__(kRowWarps * 32, 1)
+rows_tensor_codes(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg, int mode, int stat_ctas,
+                  const ScopePartial* __restrict__ partials, const SegRecord* __restrict__ recs,
+                  int8_t* __restrict__ x_q, float* __restrict__ gamma, float* __restrict__ eta) {
+  extern __shared__ __align__(16) unsigned char stage[];
+  __shared__ int counter;
+  __shared__ double gam_s[BL_MAX_GROUPS], eta_s[BL_MAX_GROUPS];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (threadIdx.x == 0) counter = 0;
+  __syncthreads();
+  const int ni = Kg / 256;
+  const int64_t first = first_segment<T>(x, segments, K, G, Kg, true, &counter, stage);   // in flight during the fold
+  for (int g = warp; g < G; g += kRowWarps) {
+    unsigned long long lo = ~0ull, hi = 0ull;
+    for (int c = lane; c < stat_ctas; c += 32) {
+      const ScopePartial p = partials[(size_t)c * G + g];
+      lo = min(lo, p.lo); hi = max(hi, p.hi);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      lo = min(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, o));
+      hi = max(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, o));
+    }
+    if (lane == 0) {
+      double gam, et;
+      scope_gamma_eta(mode, dec_ordered64(lo), dec_ordered64(hi), gam, et);
+      gam_s[g] = gam; eta_s[g] = et;
+      if (blockIdx.x == 0) {
+        gamma[g] = (float)gam;
+        if (eta) eta[g] = (float)et;
+      }
+    }
   }
+  __syncthreads();
+  for_each_segment<T>(x, segments, K, G, Kg, true, &counter, stage, first, [&](int64_t seg, const uint4* slot) {
+    const SegRecord rec = recs[seg];
+    const int g = (int)(seg % G);
+    const RowMap map = row_map(mode, rec.mean, rec.rstd, gam_s[g], eta_s[g], rec.xlo, rec.xhi);
+    row_store_codes<T>(slot, ni, lane, map, x_q + (seg / G) * K + g * (int64_t)Kg);
+  });
+}
+
+// Grid of the persistent kernels: one CTA per SM, never more CTAs than segments.
+inline cudaError_t rows_grid(int64_t segments, unsigned* grid) {
+  int dev = 0, sms = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return e;
+  int64_t g = sms < kMaxStatCtas ? sms : kMaxStatCtas;
+  if (g > segments) g = segments;
+  *grid = (unsigned)(g < 1 ? 1 : g);
+  return cudaSuccess;
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kRowWarps * 32, 2)
-rows_tensor_codes(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg, int mode,
-                  const TensorScope* __restrict__ sc, const SegRecord* __restrict__ recs,
-                  int8_t* __restrict__ x_q, float* __restrict__ gamma, float* __restrict__ eta) {
-  const int lane = threadIdx.x & 31;
-  const int64_t seg = (int64_t)blockIdx.x * kRowWarps + (threadIdx.x >> 5);
-  if (seg >= segments) return;
-  const int g = (int)(seg % G);
-  const int64_t base = (seg / G) * K + g * (int64_t)Kg;
-  const int nchunks = Kg / 8;
-  uint4 raw[kRowRegs];
-  row_load<T>(x + base, nchunks, lane, raw);                      // in flight during the scalar work below
-  const SegRecord rec = recs[seg];
-  const double lo = dec_ordered64(sc->enc_min[g]), hi = dec_ordered64(sc->enc_max[g]);
-  double gam, et;
-  scope_gamma_eta(mode, lo, hi, gam, et);
-  const RowMap map = row_map(mode, rec.mean, rec.rstd, gam, et, rec.xabs);
-  if (seg < G && lane == 0) {                                      // token 0 reports the scope's gamma / eta
-    gamma[g] = (float)gam;
-    if (eta) eta[g] = (float)et;
+cudaError_t run_rows(const QuantArgs& a, cudaStream_t s) {
+  const T* x = reinterpret_cast<const T*>(a.x);
+  const int Kg = (int)(a.K / a.G);
+  const int64_t segments = a.M * a.G;
+  const double inv_kg = 1.0 / (double)Kg;
+  constexpr int kThreads = kRowWarps * 32;
+  unsigned grid = 1;
+  cudaError_t e = rows_grid(segments, &grid);
+  if (e != cudaSuccess) return e;
+  const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+  if (a.gran == BL_PER_TOKEN) {
+    if ((e = cudaFuncSetAttribute(rows_per_token<T>, attr, kRowStage)) != cudaSuccess) return e;
+    rows_per_token<T><<<grid, kThreads, kRowStage, s>>>(x, segments, a.K, a.G, Kg, (int)a.mode, a.ln_eps, inv_kg,
+                                                        a.x_q, a.gamma, a.eta);
+    return cudaGetLastError();
   }
-  row_store_codes<T>(raw, nchunks, lane, map, x_q + base);
+  ScopePartial* partials = reinterpret_cast<ScopePartial*>(reinterpret_cast<char*>(a.ws) + sizeof(TensorScope));
+  SegRecord* recs = reinterpret_cast<SegRecord*>(reinterpret_cast<char*>(a.ws) + kWsHeaderBytes);
+  if ((e = cudaFuncSetAttribute(rows_tensor_stats<T>, attr, kRowStage)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(rows_tensor_codes<T>, attr, kRowStage)) != cudaSuccess) return e;
+  rows_tensor_stats<T><<<grid, kThreads, kRowStage, s>>>(x, segments, a.K, a.G, Kg, a.ln_eps, inv_kg, partials, recs);
+  rows_tensor_codes<T><<<grid, kThreads, kRowStage, s>>>(x, segments, a.K, a.G, Kg, (int)a.mode, (int)grid, partials,
+                                                         recs, a.x_q, a.gamma, a.eta);
+  return cudaGetLastError();
 }
 
 template <typename T>
@@ -406,23 +558,8 @@ cudaError_t run(const QuantArgs& a, cudaStream_t s) {
   const size_t smem = (size_t)Kg * sizeof(float);
   const unsigned grid = (unsigned)(a.M * a.G);
   cudaError_t e;
-  if (Kg <= RowTraits<T>::kMaxKg) {                              // a segment fits a warp's registers
-    const int64_t segments = a.M * a.G;
-    const unsigned rgrid = (unsigned)((segments + kRowWarps - 1) / kRowWarps);
-    const double inv_kg = 1.0 / (double)Kg;
-    if (a.gran == BL_PER_TOKEN) {
-      rows_per_token<T><<<rgrid, kRowWarps * 32, 0, s>>>(x, segments, a.K, a.G, (int)Kg, (int)a.mode, a.ln_eps,
-                                                         inv_kg, a.x_q, a.gamma, a.eta);
-      return cudaGetLastError();
-    }
-    TensorScope* sc = reinterpret_cast<TensorScope*>(a.ws);
-    SegRecord* recs = reinterpret_cast<SegRecord*>(reinterpret_cast<char*>(a.ws) + sizeof(TensorScope));
-    init_scope<<<1, BL_MAX_GROUPS, 0, s>>>(sc);
-    rows_tensor_stats<T><<<rgrid, kRowWarps * 32, 0, s>>>(x, segments, a.K, a.G, (int)Kg, a.ln_eps, inv_kg, sc, recs);
-    rows_tensor_codes<T><<<rgrid, kRowWarps * 32, 0, s>>>(x, segments, a.K, a.G, (int)Kg, (int)a.mode, sc, recs,
-                                                          a.x_q, a.gamma, a.eta);
-    return cudaGetLastError();
-  }
+  if (Kg % 256 == 0 && Kg <= RowTraits<T>::kMaxKg)               // whole chunks per lane, segment fits a slot
+    return run_rows<T>(a, s);
   if (a.gran == BL_PER_TOKEN) {
     if (smem > 48 * 1024) {
       e = cudaFuncSetAttribute(quant_per_token<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -433,7 +570,7 @@ cudaError_t run(const QuantArgs& a, cudaStream_t s) {
     return cudaGetLastError();
   }
   TensorScope* sc = reinterpret_cast<TensorScope*>(a.ws);
-  SegRecord* recs = reinterpret_cast<SegRecord*>(reinterpret_cast<char*>(a.ws) + sizeof(TensorScope));
+  SegRecord* recs = reinterpret_cast<SegRecord*>(reinterpret_cast<char*>(a.ws) + kWsHeaderBytes);
   if (smem > 48 * 1024) {
     e = cudaFuncSetAttribute(tensor_stats<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -447,7 +584,7 @@ cudaError_t run(const QuantArgs& a, cudaStream_t s) {
 }  // namespace
 
 size_t quant_ws_bytes(int64_t M, int G) {
-  return sizeof(TensorScope) + (size_t)M * (size_t)G * sizeof(SegRecord);
+  return kWsHeaderBytes + (size_t)M * (size_t)G * sizeof(SegRecord);
 }
 
 // ---- built-in scratch of bitlinear_quant_act_noalloc -------------------------------------------
@@ -455,7 +592,7 @@ size_t quant_ws_bytes(int64_t M, int G) {
 // The array lives in the library image: every GPU that loads the library holds these bytes until
 // the process exits.  Host code must not hand the symbol itself to a kernel (on the host the name
 // is only a stand-in); it asks the runtime for the device address once per device.
-constexpr size_t kNoAllocBytes = sizeof(TensorScope) + (size_t)BL_NOALLOC_MAX_SEGMENTS * sizeof(SegRecord);
+constexpr size_t kNoAllocBytes = kWsHeaderBytes + (size_t)BL_NOALLOC_MAX_SEGMENTS * sizeof(SegRecord);
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
 
 // Device address of the built-in scratch on the current device (cached per device ordinal).
@@ -498,8 +635,9 @@ extern "C" bl_status bitlinear_quant_act_noalloc(const void* x, bl_dtype xt, int
   void* scratch = nullptr;
   if (bl::noalloc_scratch_address(&scratch) != cudaSuccess) return BL_ERR_CUDA;
   // Same validation and the same kernels as bitlinear_quant_act, with the scratch passed as its
-  // workspace.  tensor_stats rewrites every record it later reads and init_scope resets the
-  // running extremes, so nothing of an earlier call survives into this one.
+  // workspace.  The first pass rewrites every record and every partial extreme that the second
+  // pass reads (the long-segment kernels reset their running extremes first), so nothing of an
+  // earlier call survives into this one.
   return bitlinear_quant_act(x, xt, M, K, G, b, mode, gran, ln_eps, x_q, gamma, eta, scratch,
                              bl::kNoAllocBytes, stream);
 }
