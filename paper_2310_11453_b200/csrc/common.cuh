@@ -11,6 +11,32 @@
 
 namespace bl {
 
+// Programmatic dependent launch.  A kernel launched through launch_pdl() may be scheduled while
+// the kernel before it on the stream is still running: it calls pdl_wait() before its first
+// access to global memory (after set-up that touches only its own shared memory), which blocks
+// until everything earlier on the stream has completed and is visible.  pdl_launch_dependents()
+// lets the kernel after this one be scheduled early in the same way.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t s,
+                              Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 constexpr int kQb = 128;             // Q_b = 2^(b-1), b = 8
 constexpr int kCodeMax = kQb - 1;    // Clip bound with the paper's eps taken as one code
 constexpr float kInvQb = 1.0f / 128.0f;

@@ -155,6 +155,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_rank();
   const bool leader = rank == 0;
+  pdl_launch_dependents();
 
   const uint32_t m_tiles = (uint32_t)((a.M + kPairM - 1) / kPairM), n_tiles = (uint32_t)((a.N + kBN - 1) / kBN);
   const uint32_t tiles = m_tiles * n_tiles;
@@ -176,7 +177,6 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
       mbar_init(smem_u32(&ctl->tmem_empty[b]), 8);
     }
     ctl->abort_flag = 0;
-    if (blockIdx.x == 0) *a.status = 0u;             // a timeout (seconds later) overwrites it
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 2) {
@@ -189,6 +189,10 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
   cluster_sync_all();                                // both CTAs' barriers exist before any remote arrive
   tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
+  // Everything above touched only this cluster's shared and tensor memory, so it may overlap the
+  // end of the kernel before this one on the stream; from here on global memory is read.
+  pdl_wait();
+  if (blockIdx.x == 0 && threadIdx.x == 0) *a.status = 0u;   // a timeout (seconds later) overwrites it
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer (own codes)
@@ -433,8 +437,7 @@ cudaError_t launch(const GemmArgs& a, cudaStream_t s) {
     if (resident[kMode][ti] < clusters) clusters = resident[kMode][ti];
   }
   if (tiles < clusters) clusters = tiles;
-  kern<<<(unsigned)(2 * clusters), kThreads, kSmemBytes, s>>>(map, a, (int)(box_m * kBK));
-  return cudaGetLastError();
+  return launch_pdl(kern, (unsigned)(2 * clusters), kThreads, kSmemBytes, s, map, a, (int)(box_m * kBK));
 }
 
 }  // namespace

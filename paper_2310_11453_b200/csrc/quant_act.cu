@@ -419,7 +419,9 @@ rows_per_token(const T* __restrict__ x, int64_t segments, int64_t K, int G, int 
   __shared__ int counter;
   const int lane = threadIdx.x & 31;
   if (threadIdx.x == 0) counter = 0;
+  pdl_launch_dependents();
   __syncthreads();
+  pdl_wait();
   const int ni = Kg / 256;
   const int64_t first = first_segment<T>(x, segments, K, G, Kg, false, &counter, stage);
   for_each_segment<T>(x, segments, K, G, Kg, false, &counter, stage, first, [&](int64_t seg, const uint4* slot) {
@@ -449,7 +451,9 @@ rows_tensor_stats(const T* __restrict__ x, int64_t segments, int64_t K, int G, i
   const int lane = threadIdx.x & 31;
   if (threadIdx.x == 0) counter = 0;
   if (threadIdx.x < BL_MAX_GROUPS) { part_lo[threadIdx.x] = ~0ull; part_hi[threadIdx.x] = 0ull; }
+  pdl_launch_dependents();
   __syncthreads();
+  pdl_wait();
   const int ni = Kg / 256;
   const int64_t first = first_segment<T>(x, segments, K, G, Kg, false, &counter, stage);
   for_each_segment<T>(x, segments, K, G, Kg, false, &counter, stage, first, [&](int64_t seg, const uint4* slot) {
@@ -478,7 +482,9 @@ rows_tensor_codes(const T* __restrict__ x, int64_t segments, int64_t K, int G, i
   __shared__ double gam_s[BL_MAX_GROUPS], eta_s[BL_MAX_GROUPS];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   if (threadIdx.x == 0) counter = 0;
+  pdl_launch_dependents();
   __syncthreads();
+  pdl_wait();
   const int ni = Kg / 256;
   const int64_t first = first_segment<T>(x, segments, K, G, Kg, true, &counter, stage);   // in flight during the fold
   for (int g = warp; g < G; g += kRowWarps) {
@@ -537,18 +543,18 @@ cudaError_t run_rows(const QuantArgs& a, cudaStream_t s) {
   const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
   if (a.gran == BL_PER_TOKEN) {
     if ((e = cudaFuncSetAttribute(rows_per_token<T>, attr, kRowStage)) != cudaSuccess) return e;
-    rows_per_token<T><<<grid, kThreads, kRowStage, s>>>(x, segments, a.K, a.G, Kg, (int)a.mode, a.ln_eps, inv_kg,
-                                                        a.x_q, a.gamma, a.eta);
-    return cudaGetLastError();
+    return launch_pdl(rows_per_token<T>, grid, kThreads, kRowStage, s, x, segments, a.K, a.G, Kg, (int)a.mode,
+                      a.ln_eps, inv_kg, a.x_q, a.gamma, a.eta);
   }
   ScopePartial* partials = reinterpret_cast<ScopePartial*>(reinterpret_cast<char*>(a.ws) + sizeof(TensorScope));
   SegRecord* recs = reinterpret_cast<SegRecord*>(reinterpret_cast<char*>(a.ws) + kWsHeaderBytes);
   if ((e = cudaFuncSetAttribute(rows_tensor_stats<T>, attr, kRowStage)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(rows_tensor_codes<T>, attr, kRowStage)) != cudaSuccess) return e;
-  rows_tensor_stats<T><<<grid, kThreads, kRowStage, s>>>(x, segments, a.K, a.G, Kg, a.ln_eps, inv_kg, partials, recs);
-  rows_tensor_codes<T><<<grid, kThreads, kRowStage, s>>>(x, segments, a.K, a.G, Kg, (int)a.mode, (int)grid, partials,
-                                                         recs, a.x_q, a.gamma, a.eta);
-  return cudaGetLastError();
+  e = launch_pdl(rows_tensor_stats<T>, grid, kThreads, kRowStage, s, x, segments, a.K, a.G, Kg, a.ln_eps, inv_kg,
+                 partials, recs);
+  if (e != cudaSuccess) return e;
+  return launch_pdl(rows_tensor_codes<T>, grid, kThreads, kRowStage, s, x, segments, a.K, a.G, Kg, (int)a.mode,
+                    (int)grid, (const ScopePartial*)partials, (const SegRecord*)recs, a.x_q, a.gamma, a.eta);
 }
 
 template <typename T>
