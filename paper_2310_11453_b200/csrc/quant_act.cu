@@ -352,9 +352,17 @@ __device__ __forceinline__ RowRange cta_range(int64_t segments) {
   r.end = segments * ((int64_t)blockIdx.x + 1) / (int64_t)gridDim.x;
   return r;
 }
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
-               "l"(gsrc) : "memory");
+// 16-byte asynchronous copy with an L2 eviction policy for the line it reads.
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc, uint64_t policy) {
+  asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;"
+               ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc), "l"(policy) : "memory");
+}
+// keep = true: the lines are read again soon (first per-tensor pass); false: this is their last use.
+__device__ __forceinline__ uint64_t l2_policy(bool keep) {
+  uint64_t p;
+  if (keep) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  else asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 // All of this thread's copy groups but the newest are complete; __syncwarp() makes the other
@@ -367,7 +375,7 @@ __device__ __forceinline__ void cp_async_wait_but_newest() { asm volatile("cp.as
 // first pass read last, the ones most likely still in L2.
 template <typename T>
 __device__ __forceinline__ int64_t stage_next(const T* __restrict__ x, const RowRange& rg, int64_t K, int G, int Kg,
-                                              bool reverse, int* counter, uint4* slot, int lane) {
+                                              bool reverse, uint64_t policy, int* counter, uint4* slot, int lane) {
   int r = 0;
   if (lane == 0) r = atomicAdd(counter, 1);
   r = __shfl_sync(0xFFFFFFFFu, r, 0);
@@ -377,7 +385,7 @@ __device__ __forceinline__ int64_t stage_next(const T* __restrict__ x, const Row
     const uint4* src = reinterpret_cast<const uint4*>(x + (seg / G) * K + (seg % G) * (int64_t)Kg);
     const int nv = Kg / 256 * RowTraits<T>::kVecPerChunk;      // 16-byte pieces per lane
 #pragma unroll 4
-    for (int i = 0; i < nv; ++i) cp_async16(slot + lane + 32 * i, src + lane + 32 * i);
+    for (int i = 0; i < nv; ++i) cp_async16(slot + lane + 32 * i, src + lane + 32 * i, policy);
   }
   cp_async_commit();
   return seg;
@@ -387,15 +395,16 @@ __device__ __forceinline__ int64_t stage_next(const T* __restrict__ x, const Row
 // the next one already on its way.
 template <typename T, typename Body>
 __device__ __forceinline__ void for_each_segment(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg,
-                                                 bool reverse, int* counter, unsigned char* stage, int64_t first_seg,
-                                                 Body body) {
+                                                 bool reverse, uint64_t policy, int* counter, unsigned char* stage,
+                                                 int64_t first_seg, Body body) {
   const int lane = threadIdx.x & 31;
   uint4* slots = reinterpret_cast<uint4*>(stage + (size_t)(threadIdx.x >> 5) * 2 * kSlotBytes);
   const RowRange rg = cta_range(segments);
   int cur = 0;
   int64_t seg = first_seg;
   while (seg >= 0) {
-    const int64_t next = stage_next<T>(x, rg, K, G, Kg, reverse, counter, slots + (cur ^ 1) * (kSlotBytes / 16), lane);
+    const int64_t next =
+        stage_next<T>(x, rg, K, G, Kg, reverse, policy, counter, slots + (cur ^ 1) * (kSlotBytes / 16), lane);
     cp_async_wait_but_newest();
     __syncwarp();
     body(seg, slots + cur * (kSlotBytes / 16));
@@ -406,9 +415,9 @@ __device__ __forceinline__ void for_each_segment(const T* __restrict__ x, int64_
 // First draw of a warp (into slot 0), split off so that a kernel can put work between it and the loop.
 template <typename T>
 __device__ __forceinline__ int64_t first_segment(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg,
-                                                 bool reverse, int* counter, unsigned char* stage) {
+                                                 bool reverse, uint64_t policy, int* counter, unsigned char* stage) {
   uint4* slots = reinterpret_cast<uint4*>(stage + (size_t)(threadIdx.x >> 5) * 2 * kSlotBytes);
-  return stage_next<T>(x, cta_range(segments), K, G, Kg, reverse, counter, slots, threadIdx.x & 31);
+  return stage_next<T>(x, cta_range(segments), K, G, Kg, reverse, policy, counter, slots, threadIdx.x & 31);
 }
 
 template <typename T>
@@ -423,8 +432,9 @@ rows_per_token(const T* __restrict__ x, int64_t segments, int64_t K, int G, int 
   __syncthreads();
   pdl_wait();
   const int ni = Kg / 256;
-  const int64_t first = first_segment<T>(x, segments, K, G, Kg, false, &counter, stage);
-  for_each_segment<T>(x, segments, K, G, Kg, false, &counter, stage, first, [&](int64_t seg, const uint4* slot) {
+  const uint64_t pol = l2_policy(false);
+  const int64_t first = first_segment<T>(x, segments, K, G, Kg, false, pol, &counter, stage);
+  for_each_segment<T>(x, segments, K, G, Kg, false, pol, &counter, stage, first, [&](int64_t seg, const uint4* slot) {
     const RowStats st = row_stats<T>(slot, ni, lane, ln_eps, inv_kg);
     const double lo = ((double)st.xlo - st.mean) * st.rstd, hi = ((double)st.xhi - st.mean) * st.rstd;
     double gam, et;
@@ -455,8 +465,9 @@ rows_tensor_stats(const T* __restrict__ x, int64_t segments, int64_t K, int G, i
   __syncthreads();
   pdl_wait();
   const int ni = Kg / 256;
-  const int64_t first = first_segment<T>(x, segments, K, G, Kg, false, &counter, stage);
-  for_each_segment<T>(x, segments, K, G, Kg, false, &counter, stage, first, [&](int64_t seg, const uint4* slot) {
+  const uint64_t pol = l2_policy(true);                  // the second pass reads x again
+  const int64_t first = first_segment<T>(x, segments, K, G, Kg, false, pol, &counter, stage);
+  for_each_segment<T>(x, segments, K, G, Kg, false, pol, &counter, stage, first, [&](int64_t seg, const uint4* slot) {
     const RowStats st = row_stats<T>(slot, ni, lane, ln_eps, inv_kg);
     if (lane == 0) {
       const int g = (int)(seg % G);
@@ -486,7 +497,8 @@ rows_tensor_codes(const T* __restrict__ x, int64_t segments, int64_t K, int G, i
   __syncthreads();
   pdl_wait();
   const int ni = Kg / 256;
-  const int64_t first = first_segment<T>(x, segments, K, G, Kg, true, &counter, stage);   // in flight during the fold
+  const uint64_t pol = l2_policy(false);
+  const int64_t first = first_segment<T>(x, segments, K, G, Kg, true, pol, &counter, stage);   // in flight during the fold
   for (int g = warp; g < G; g += kRowWarps) {
     unsigned long long lo = ~0ull, hi = 0ull;
     for (int c = lane; c < stat_ctas; c += 32) {
@@ -509,7 +521,7 @@ rows_tensor_codes(const T* __restrict__ x, int64_t segments, int64_t K, int G, i
     }
   }
   __syncthreads();
-  for_each_segment<T>(x, segments, K, G, Kg, true, &counter, stage, first, [&](int64_t seg, const uint4* slot) {
+  for_each_segment<T>(x, segments, K, G, Kg, true, pol, &counter, stage, first, [&](int64_t seg, const uint4* slot) {
     const SegRecord rec = recs[seg];
     const int g = (int)(seg % G);
     const RowMap map = row_map(mode, rec.mean, rec.rstd, gam_s[g], eta_s[g], rec.xlo, rec.xhi);
