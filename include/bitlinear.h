@@ -178,6 +178,46 @@ bl_status bitlinear_matmul_dequant(const int8_t* x_q, int64_t M, int64_t K, int6
                                    const float* beta, const int32_t* rowsum, void* y, bl_dtype yt,
                                    void* ws, size_t ws_bytes, void* stream);
 
+/* bitlinear_matmul_dequant with output-side options, for fusing what follows a BitLinear in the
+ * decoder block (Sec. 2, Fig. 2b) into its epilogue, and for weights whose alpha / beta are taken
+ * per block of output features (the partitioning of Sec. 2.1 "Model parallelism with Group
+ * Quantization", Eq. 13, applied along N: each device's slice of output features carries its own
+ * alpha and beta; also how W_q, W_k, W_v stacked into one [3d, d] matrix keep their own beta).
+ *   beta_rows  output features per beta block: beta is [N / beta_rows, G] (block-major), rowsum
+ *              stays [N, G].  0 means one block (beta [G]).  Must divide N and be a multiple of 32.
+ *   relu       non-zero: y = max(y, 0), applied before the residual.
+ *   residual   NULL or [M, N] of dtype yt with row stride ld_res (elements): y += residual.
+ *              May alias y only if ld_res == ld_y and residual == y (each element is read by
+ *              the thread that then writes it).
+ *   ld_y       row stride of y in elements (0 means N), so y may be a column block of a wider buffer.
+ * With epi == NULL or all-zero options the call equals bitlinear_matmul_dequant. */
+typedef struct {
+  int64_t beta_rows;
+  int relu;
+  const void* residual;
+  int64_t ld_res;
+  int64_t ld_y;
+} bl_epilogue;
+bl_status bitlinear_matmul_dequant_ex(const int8_t* x_q, int64_t M, int64_t K, int64_t N, int G,
+                                      bl_gran gran, const float* gamma, const float* eta,
+                                      int eta_correction, const uint8_t* W_packed, bl_layout layout,
+                                      const float* beta, const int32_t* rowsum, const bl_epilogue* epi,
+                                      void* y, bl_dtype yt, void* ws, size_t ws_bytes, void* stream);
+
+/* bitlinear_binarize_pack for NB blocks of N / NB consecutive output features, each with its own
+ * alpha_g and beta_g (Eq. 13 applied along N, see bitlinear_matmul_dequant_ex): block j is
+ * binarised against the mean of its own rows.
+ *   alpha, beta  [NB, G];  alpha_in NULL or [NB, G];  rowsum NULL or [N, G].
+ *   W_packed     the blocks' packed images one after the other, which for PREFILL (N / NB a
+ *                multiple of 128) and CANONICAL / DECODE layouts is the packed image of the
+ *                whole [N, K] matrix.
+ * Runs one pass of bitlinear_binarize_pack per block on `stream`; the workspace is that of one
+ * block (BL_OP_BINARIZE_PACK), reused in stream order. */
+bl_status bitlinear_binarize_pack_nsplit(const void* W, bl_dtype wt, int64_t N, int64_t K, int G, int NB,
+                                         bl_layout layout, const float* alpha_in, uint8_t* W_packed,
+                                         float* alpha, float* beta, int32_t* rowsum, void* ws,
+                                         size_t ws_bytes, void* stream);
+
 /* Steps 1, 2, 4 for one token (M = 1), fused in a single kernel that streams the packed
  * weights once; Eq. 11 with per-token gamma.  W_packed must be in DECODE layout.
  *   x [K] of dtype xt;  y [N] of dtype yt.  No workspace, no device-side waits. */
@@ -207,7 +247,13 @@ bl_status bitlinear_attention_causal(const void* q, const void* k, const void* v
  * All weight buffers are PREFILL-packed with one group: W_q, W_k, W_v, W_o [d,d], W_up [ffn,d],
  * W_down [d,ffn]; beta_* point to one float each (as written by bitlinear_binarize_pack).
  * Every intermediate is a caller buffer (fp16, row-major), so each stage can be inspected:
- *   q, k, v, a, h [T,d];  u [T,ffn];  y [T,d] (also used for the two projection outputs).
+ *   q, k, v [T,d] with row stride ld_qkv (0 means d);  a, h [T,d];  u [T,ffn];  y [T,d].
+ * ReLU and the two residual adds run in the epilogues of the up, O and down GEMMs.  Q, K and V run
+ * as ONE GEMM over a [3d, d] weight matrix when the caller lays them out for it: W_k directly
+ * behind W_q and W_v behind W_k in memory (likewise beta_q, beta_k, beta_v, as written by
+ * bitlinear_binarize_pack_nsplit with NB = 3), and q, k, v the three column blocks of one
+ * [T, 3d] buffer (k = q + d, v = q + 2d, ld_qkv = 3d); otherwise as three GEMMs.  The values
+ * written are the same either way.  9 launches in the fused layout, 11 otherwise.
  * Workspace: BL_OP_BLOCK_FORWARD (codes, gamma, eta, quant and GEMM scratch).  Asynchronous on
  * `stream`; bitlinear_ws_status(ws, stream) reports a device-side timeout of the GEMMs. */
 typedef struct {
@@ -216,6 +262,7 @@ typedef struct {
 } bl_block_weights;
 typedef struct {
   void *q, *k, *v, *a, *h, *u;
+  int64_t ld_qkv;
 } bl_block_buffers;
 bl_status bitlinear_block_forward(const void* x, int batch, int seq, int heads, int64_t ffn, float ln_eps,
                                   const bl_block_weights* w, const bl_block_buffers* buf, void* y, void* ws,

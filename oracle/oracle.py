@@ -53,6 +53,36 @@ def binarize(W, G=1, alpha_in=None):
     return dict(bits=bits, alpha=alpha, beta=beta, rowsum=rowsum)
 
 
+def binarize_nsplit(W, NB, G=1, alpha_in=None):
+    """Eq. 13 with the partition taken along the output features (Sec. 2.1, model parallelism with
+    group quantisation): NB blocks of N/NB consecutive rows, each binarised against its own
+    alpha_g and scaled by its own beta_g.  Returns bits [N,K/8], alpha, beta [NB,G], rowsum [N,G]."""
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    N, K = W.shape
+    if N % NB != 0:
+        raise ValueError("NB must divide N")
+    rows = N // NB
+    parts = [binarize(W[j * rows:(j + 1) * rows], G=G,
+                      alpha_in=None if alpha_in is None else np.asarray(alpha_in)[j]) for j in range(NB)]
+    return dict(bits=np.concatenate([p["bits"] for p in parts], axis=0),
+                alpha=np.stack([p["alpha"] for p in parts]), beta=np.stack([p["beta"] for p in parts]),
+                rowsum=np.concatenate([p["rowsum"] for p in parts], axis=0))
+
+
+def dequant_nsplit(acc, beta, gamma, gran=PER_TOKEN, eta=None, rowsum=None, eta_correction=False):
+    """Eq. 11 rescale with beta [NB,G] per block of output features.  acc [G,M,N]; returns y f64 [M,N]."""
+    beta = np.asarray(beta, dtype=np.float64)
+    NB = beta.shape[0]
+    G, M, N = acc.shape
+    rows = N // NB
+    cols = []
+    for j in range(NB):
+        sl = slice(j * rows, (j + 1) * rows)
+        cols.append(dequant(acc[:, :, sl], beta[j], gamma, gran=gran, eta=eta,
+                            rowsum=None if rowsum is None else rowsum[sl], eta_correction=eta_correction))
+    return np.concatenate(cols, axis=1)
+
+
 def quant_act(x, G=1, mode=ABSMAX, gran=PER_TOKEN, ln_eps=1e-5, want_xhat=False):
     """Eq. 12/15 then Eq. 4-6/14.  Returns dict(codes i8 [M,K], gamma, eta f64, xhat?)."""
     x = np.ascontiguousarray(x, dtype=np.float32)

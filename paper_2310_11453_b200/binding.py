@@ -21,13 +21,14 @@ CANONICAL, PREFILL, DECODE = 0, 1, 2
 OP_BINARIZE_PACK, OP_QUANT_ACT, OP_FORWARD, OP_MATMUL_I32, OP_MATMUL_DEQUANT, OP_BLOCK_FORWARD = 0, 1, 2, 3, 4, 5
 MAX_GROUPS = 64
 NOALLOC_MAX_SEGMENTS = 16384
-ERR_TOO_LARGE = 8
+ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_TOO_LARGE = 1, 2, 3, 4, 5, 6, 7, 8
 
 EXPORTS = [
     "bitlinear_status_string", "bitlinear_workspace_bytes", "bitlinear_packed_bytes",
     "bitlinear_layout_index", "bitlinear_binarize_pack", "bitlinear_quant_act", "bitlinear_quant_act_noalloc",
     "bitlinear_forward", "bitlinear_matmul_i32", "bitlinear_matmul_dequant", "bitlinear_gemv_decode",
     "bitlinear_attention_causal", "bitlinear_block_forward", "bitlinear_ws_status",
+    "bitlinear_matmul_dequant_ex", "bitlinear_binarize_pack_nsplit",
 ]
 
 _DTYPES = {torch.float32: F32, torch.float16: F16, torch.bfloat16: BF16}
@@ -80,6 +81,11 @@ def lib():
         L.bitlinear_block_forward.argtypes = [vp, ci, ci, ci, i64, C.c_float, vp, vp, vp, vp, sz, vp]
         L.bitlinear_ws_status.restype = ci
         L.bitlinear_ws_status.argtypes = [vp, vp]
+        L.bitlinear_matmul_dequant_ex.restype = ci
+        L.bitlinear_matmul_dequant_ex.argtypes = [vp, i64, i64, i64, ci, ci, vp, vp, ci, vp, ci, vp, vp, vp, vp, ci,
+                                                  vp, sz, vp]
+        L.bitlinear_binarize_pack_nsplit.restype = ci
+        L.bitlinear_binarize_pack_nsplit.argtypes = [vp, ci, i64, i64, ci, ci, ci, vp, vp, vp, vp, vp, vp, sz, vp]
         _lib = L
     return _lib
 
@@ -151,6 +157,26 @@ def binarize_pack(W, G=1, layout=CANONICAL, alpha_in=None, want_rowsum=True, out
                                          _stream())
     _check(code, "bitlinear_binarize_pack")
     return dict(W_packed=packed, alpha=alpha, beta=beta, rowsum=rowsum, layout=layout, N=N, K=K, G=G)
+
+
+def binarize_pack_nsplit(W, NB, G=1, layout=CANONICAL, alpha_in=None, want_rowsum=True, ws=None):
+    """bitlinear_binarize_pack_nsplit.  W [N,K]; NB blocks of N/NB output features, each with its own
+    alpha / beta.  Returns dict(W_packed, alpha, beta [NB,G], rowsum [N,G] or None, beta_rows)."""
+    N, K = W.shape
+    dev = W.device
+    rows = N // NB
+    nbytes = NB * packed_bytes(layout, rows, K)
+    packed = torch.empty(max(nbytes, 16), dtype=torch.uint8, device=dev)
+    alpha = torch.empty((NB, G), dtype=torch.float32, device=dev)
+    beta = torch.empty((NB, G), dtype=torch.float32, device=dev)
+    rowsum = torch.empty((N, G), dtype=torch.int32, device=dev) if want_rowsum else None
+    ws = _ws(workspace_bytes(OP_BINARIZE_PACK, 1, rows, K, G), dev, ws)
+    code = lib().bitlinear_binarize_pack_nsplit(_ptr(W), _dt(W), N, K, G, NB, layout, _ptr(alpha_in), _ptr(packed),
+                                                _ptr(alpha), _ptr(beta), _ptr(rowsum), _ptr(ws), ws.numel(),
+                                                _stream())
+    _check(code, "bitlinear_binarize_pack_nsplit")
+    return dict(W_packed=packed, alpha=alpha, beta=beta, rowsum=rowsum, layout=layout, N=N, K=K, G=G, NB=NB,
+                beta_rows=rows)
 
 
 def quant_act(x, G=1, mode=ABSMAX, gran=PER_TOKEN, ln_eps=1e-5, b=8, out=None, ws=None):
@@ -227,6 +253,32 @@ def matmul_dequant(x_q, gamma, W_packed, beta, N, G=1, gran=PER_TOKEN, layout=CA
     return y
 
 
+class _Epilogue(C.Structure):
+    _fields_ = [("beta_rows", C.c_int64), ("relu", C.c_int), ("residual", C.c_void_p), ("ld_res", C.c_int64),
+                ("ld_y", C.c_int64)]
+
+
+def matmul_dequant_ex(x_q, gamma, W_packed, beta, N, G=1, gran=PER_TOKEN, layout=CANONICAL, eta=None,
+                      rowsum=None, eta_correction=False, beta_rows=0, relu=False, residual=None, y=None,
+                      out_dtype=torch.float32, ws=None):
+    """bitlinear_matmul_dequant_ex.  `y` may be a column slice of a wider row-major tensor (its row
+    stride becomes ld_y), `residual` likewise.  Returns y [M,N]."""
+    M, K = x_q.shape
+    dev = x_q.device
+    if y is None:
+        y = torch.empty((M, N), dtype=out_dtype, device=dev)
+    assert y.stride(1) == 1 and (residual is None or (residual.stride(1) == 1 and residual.dtype == y.dtype))
+    epi = _Epilogue(int(beta_rows), 1 if relu else 0, _ptr(residual),
+                    residual.stride(0) if residual is not None else 0, y.stride(0))
+    ws = _ws(workspace_bytes(OP_MATMUL_DEQUANT, M, N, K, G), dev, ws)
+    code = lib().bitlinear_matmul_dequant_ex(_ptr(x_q), M, K, N, G, gran, _ptr(gamma), _ptr(eta),
+                                             1 if eta_correction else 0, _ptr(W_packed), layout, _ptr(beta),
+                                             _ptr(rowsum), C.byref(epi), _ptr(y), _dt(y), _ptr(ws), ws.numel(),
+                                             _stream())
+    _check(code, "bitlinear_matmul_dequant_ex")
+    return y
+
+
 def gemv_decode(x, W_packed, beta, N, G=1, mode=ABSMAX, ln_eps=1e-5, rowsum=None,
                 eta_correction=False, out_dtype=None, b=8, y=None):
     """bitlinear_gemv_decode.  x [K] or [1,K]; W_packed in DECODE layout; returns y [N]."""
@@ -246,7 +298,7 @@ class _BlockWeights(C.Structure):
 
 
 class _BlockBuffers(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("q", "k", "v", "a", "h", "u")]
+    _fields_ = [(n, C.c_void_p) for n in ("q", "k", "v", "a", "h", "u")] + [("ld_qkv", C.c_int64)]
 
 
 def attention_causal(q, k, v, batch, seq, heads, head_dim=128, o=None):
@@ -262,18 +314,38 @@ def attention_causal(q, k, v, batch, seq, heads, head_dim=128, o=None):
     return o
 
 
-def block_forward(x, weights, batch, seq, heads, ffn, ln_eps=1e-5, ws=None):
+def fuse_qkv_weights(weights):
+    """Copies the packed W_q, W_k, W_v and their betas back to back (the layout that lets
+    bitlinear_block_forward run them as one GEMM); returns a new weights dict sharing the rest."""
+    q, k, v = (weights[n] for n in ("q", "k", "v"))
+    nb = packed_bytes(PREFILL, q["N"], q["K"])
+    packed = torch.cat([t["W_packed"][:nb] for t in (q, k, v)])
+    beta = torch.cat([t["beta"].reshape(1) for t in (q, k, v)])
+    fused = dict(weights)
+    for i, n in enumerate(("q", "k", "v")):
+        fused[n] = dict(weights[n], W_packed=packed[i * nb:(i + 1) * nb], beta=beta[i:i + 1])
+    fused["_qkv_storage"] = (packed, beta)
+    return fused
+
+
+def block_forward(x, weights, batch, seq, heads, ffn, ln_eps=1e-5, ws=None, fused_qkv=False):
     """bitlinear_block_forward.  x fp16 [batch*seq, heads*128]; `weights` maps q, k, v, o, up, down to
-    the dicts returned by binarize_pack(layout=PREFILL).  Returns dict(y, q, k, v, a, h, u): the output
-    and every intermediate, all fp16."""
+    the dicts returned by binarize_pack(layout=PREFILL) (pass them through fuse_qkv_weights and set
+    fused_qkv for the one-GEMM Q/K/V layout).  Returns dict(y, q, k, v, a, h, u): the output and every
+    intermediate, all fp16 (q, k, v are column slices of one [T,3d] tensor when fused_qkv)."""
     T, d = x.shape
     dev = x.device
     f16 = dict(dtype=torch.float16, device=dev)
-    out = {n: torch.empty((T, d), **f16) for n in ("q", "k", "v", "a", "h", "y")}
+    out = {n: torch.empty((T, d), **f16) for n in ("a", "h", "y")}
+    if fused_qkv:
+        qkv = torch.empty((T, 3 * d), **f16)
+        out.update(q=qkv[:, :d], k=qkv[:, d:2 * d], v=qkv[:, 2 * d:], qkv=qkv)
+    else:
+        out.update({n: torch.empty((T, d), **f16) for n in ("q", "k", "v")})
     out["u"] = torch.empty((T, ffn), **f16)
     w = _BlockWeights(*[weights[n]["W_packed"].data_ptr() for n in ("q", "k", "v", "o", "up", "down")],
                       *[weights[n]["beta"].data_ptr() for n in ("q", "k", "v", "o", "up", "down")])
-    b = _BlockBuffers(*[out[n].data_ptr() for n in ("q", "k", "v", "a", "h", "u")])
+    b = _BlockBuffers(*[out[n].data_ptr() for n in ("q", "k", "v", "a", "h", "u")], out["q"].stride(0))
     ws = _ws(workspace_bytes(OP_BLOCK_FORWARD, T, ffn, d, 1), dev, ws)
     code = lib().bitlinear_block_forward(_ptr(x), batch, seq, heads, ffn, float(ln_eps), C.byref(w), C.byref(b),
                                          _ptr(out["y"]), _ptr(ws), ws.numel(), _stream())

@@ -31,7 +31,7 @@ struct BlockWs {                       // carving of the BL_OP_BLOCK_FORWARD wor
 BlockWs carve_block(int64_t T, int64_t d, int64_t ffn) {
   BlockWs w;
   size_t off = 0;
-  const int64_t widest = ffn > d ? ffn : d;
+  const int64_t widest = ffn > 3 * d ? ffn : 3 * d;       // Q, K, V may run as one [3d, d] GEMM
   w.gemm = off;  off += gemm_ws_total(T, widest, 1);
   w.codes = off; off += round256((size_t)T * (size_t)widest);
   w.gamma = off; off += round256((size_t)T * sizeof(float));
@@ -181,11 +181,11 @@ bl_status bitlinear_matmul_i32(const int8_t* x_q, int64_t M, int64_t K, int64_t 
   return e == cudaSuccess ? BL_OK : BL_ERR_CUDA;
 }
 
-bl_status bitlinear_matmul_dequant(const int8_t* x_q, int64_t M, int64_t K, int64_t N, int G,
-                                   bl_gran gran, const float* gamma, const float* eta,
-                                   int eta_correction, const uint8_t* W_packed, bl_layout layout,
-                                   const float* beta, const int32_t* rowsum, void* y, bl_dtype yt,
-                                   void* ws, size_t ws_bytes, void* stream) {
+bl_status bitlinear_matmul_dequant_ex(const int8_t* x_q, int64_t M, int64_t K, int64_t N, int G,
+                                      bl_gran gran, const float* gamma, const float* eta,
+                                      int eta_correction, const uint8_t* W_packed, bl_layout layout,
+                                      const float* beta, const int32_t* rowsum, const bl_epilogue* epi,
+                                      void* y, bl_dtype yt, void* ws, size_t ws_bytes, void* stream) {
   if (!x_q || !W_packed || !beta || !gamma || !y) return BL_ERR_NULL;
   if (eta_correction && (!rowsum || !eta)) return BL_ERR_NULL;
   if (M <= 0 || N <= 0) return BL_ERR_SHAPE;
@@ -195,7 +195,12 @@ bl_status bitlinear_matmul_dequant(const int8_t* x_q, int64_t M, int64_t K, int6
   if (gran != BL_PER_TENSOR && gran != BL_PER_TOKEN) return BL_ERR_UNSUPPORTED;
   st = check_layout_for_gemm(layout, M, K, N, G);
   if (st != BL_OK) return st;
-  if (!aligned16(x_q) || !aligned16(W_packed) || !aligned16(y)) return BL_ERR_ALIGN;
+  bl_epilogue o{};
+  if (epi) o = *epi;
+  if (o.beta_rows < 0 || (o.beta_rows > 0 && (N % o.beta_rows != 0 || o.beta_rows % 32 != 0))) return BL_ERR_SHAPE;
+  if (o.ld_y < 0 || (o.ld_y > 0 && o.ld_y < N)) return BL_ERR_SHAPE;
+  if (o.residual && o.ld_res < N) return BL_ERR_SHAPE;
+  if (!aligned16(x_q) || !aligned16(W_packed) || !aligned16(y) || !aligned16(o.residual)) return BL_ERR_ALIGN;
   if (!ws || ws_bytes < gemm_ws_total(M, N, G)) return BL_ERR_WORKSPACE;
   if (!aligned16(ws)) return BL_ERR_ALIGN;
   cudaStream_t s = (cudaStream_t)stream;
@@ -205,10 +210,42 @@ bl_status bitlinear_matmul_dequant(const int8_t* x_q, int64_t M, int64_t K, int6
   a.x_q = x_q; a.M = M; a.K = K; a.N = N; a.G = G; a.W_packed = W_packed; a.acc = nullptr;
   a.y = y; a.yt = yt; a.beta = beta; a.gamma = gamma; a.eta = eta; a.gran = gran;
   a.rowsum = rowsum; a.eta_correction = eta_correction ? 1 : 0;
+  a.beta_rows = o.beta_rows; a.relu = o.relu ? 1 : 0; a.residual = o.residual; a.ld_res = o.ld_res; a.ld_y = o.ld_y;
   a.status = reinterpret_cast<uint32_t*>(ws);
   a.scratch = reinterpret_cast<char*>(ws) + kStatusBytes;
   cudaError_t e = (layout == BL_LAYOUT_PREFILL) ? launch_gemm_tc(a, s) : launch_gemm_simple(a, s);
   return e == cudaSuccess ? BL_OK : BL_ERR_CUDA;
+}
+
+bl_status bitlinear_matmul_dequant(const int8_t* x_q, int64_t M, int64_t K, int64_t N, int G,
+                                   bl_gran gran, const float* gamma, const float* eta,
+                                   int eta_correction, const uint8_t* W_packed, bl_layout layout,
+                                   const float* beta, const int32_t* rowsum, void* y, bl_dtype yt,
+                                   void* ws, size_t ws_bytes, void* stream) {
+  return bitlinear_matmul_dequant_ex(x_q, M, K, N, G, gran, gamma, eta, eta_correction, W_packed, layout, beta,
+                                     rowsum, nullptr, y, yt, ws, ws_bytes, stream);
+}
+
+bl_status bitlinear_binarize_pack_nsplit(const void* W, bl_dtype wt, int64_t N, int64_t K, int G, int NB,
+                                         bl_layout layout, const float* alpha_in, uint8_t* W_packed,
+                                         float* alpha, float* beta, int32_t* rowsum, void* ws,
+                                         size_t ws_bytes, void* stream) {
+  if (NB <= 0 || N <= 0 || N % NB != 0) return BL_ERR_SHAPE;
+  if (!valid_dtype(wt)) return BL_ERR_UNSUPPORTED;
+  const int64_t rows = N / NB;
+  if (layout == BL_LAYOUT_PREFILL && NB > 1 && rows % 128 != 0) return BL_ERR_SHAPE;
+  const size_t block_bytes = bitlinear_packed_bytes(layout, rows, K);
+  if (block_bytes == 0) return BL_ERR_SHAPE;
+  const size_t esz = wt == BL_F32 ? 4 : 2;
+  for (int j = 0; j < NB; ++j) {
+    const bl_status st = bitlinear_binarize_pack(
+        reinterpret_cast<const char*>(W) + (size_t)j * (size_t)rows * (size_t)K * esz, wt, rows, K, G, layout,
+        alpha_in ? alpha_in + (size_t)j * G : nullptr, W_packed ? W_packed + (size_t)j * block_bytes : nullptr,
+        alpha ? alpha + (size_t)j * G : nullptr, beta ? beta + (size_t)j * G : nullptr,
+        rowsum ? rowsum + (size_t)j * (size_t)rows * G : nullptr, ws, ws_bytes, stream);
+    if (st != BL_OK) return st;
+  }
+  return BL_OK;
 }
 
 bl_status bitlinear_forward(const void* x, bl_dtype xt, int64_t M, int64_t K, int64_t N, int G,
@@ -295,6 +332,8 @@ bl_status bitlinear_block_forward(const void* x, int batch, int seq, int heads, 
   const void* ptrs[] = {x, y, buf->q, buf->k, buf->v, buf->a, buf->h, buf->u, w->W_q, w->W_k, w->W_v, w->W_o,
                         w->W_up, w->W_down};
   for (const void* p : ptrs) if (!aligned16(p)) return BL_ERR_ALIGN;
+  const int64_t ld_qkv = buf->ld_qkv > 0 ? buf->ld_qkv : d;
+  if (ld_qkv < d || ld_qkv % 8 != 0) return BL_ERR_SHAPE;
   const BlockWs c = carve_block(T, d, ffn);
   if (!ws || ws_bytes < c.total) return BL_ERR_WORKSPACE;
   if (!aligned16(ws)) return BL_ERR_ALIGN;
@@ -309,24 +348,37 @@ bl_status bitlinear_block_forward(const void* x, int batch, int seq, int heads, 
     QuantArgs q{in, BL_F16, T, K, 1, mode, BL_PER_TOKEN, ln_eps, codes, gamma, eta, nullptr};
     return launch_quant_act(q, s) == cudaSuccess;
   };
-  auto matmul = [&](int64_t K, int64_t N, const uint8_t* W, const float* beta, void* out) -> bool {
+  // out [T,N] (row stride ld) = [relu] BitLinear(codes) [+ res]; beta holds one entry per beta_rows features.
+  auto matmul = [&](int64_t K, int64_t N, const uint8_t* W, const float* beta, int64_t beta_rows, void* out,
+                    int64_t ld, bool relu, const void* res) -> bool {
     GemmArgs g{};
     g.x_q = codes; g.M = T; g.K = K; g.N = N; g.G = 1; g.W_packed = W; g.acc = nullptr; g.y = out; g.yt = BL_F16;
     g.beta = beta; g.gamma = gamma; g.eta = eta; g.gran = BL_PER_TOKEN; g.rowsum = nullptr; g.eta_correction = 0;
+    g.beta_rows = beta_rows; g.relu = relu ? 1 : 0; g.residual = res; g.ld_res = d; g.ld_y = ld;
     g.status = reinterpret_cast<uint32_t*>(base + c.gemm);
     g.scratch = base + c.gemm + kStatusBytes;
     return launch_gemm_tc(g, s) == cudaSuccess;
   };
-  bool ok = quant(x, d, BL_ABSMAX)
-      && matmul(d, d, w->W_q, w->beta_q, buf->q) && matmul(d, d, w->W_k, w->beta_k, buf->k)
-      && matmul(d, d, w->W_v, w->beta_v, buf->v)
-      && launch_attention_causal(buf->q, buf->k, buf->v, buf->a, batch, seq, heads, d, d, s) == cudaSuccess
-      && quant(buf->a, d, BL_ABSMAX) && matmul(d, d, w->W_o, w->beta_o, buf->h)
-      && launch_add_inplace(buf->h, x, T * d, s) == cudaSuccess
-      && quant(buf->h, d, BL_ABSMAX) && matmul(d, ffn, w->W_up, w->beta_up, buf->u)
-      && launch_relu_inplace(buf->u, T * ffn, s) == cudaSuccess
-      && quant(buf->u, ffn, BL_ETA) && matmul(ffn, d, w->W_down, w->beta_down, y)
-      && launch_add_inplace(y, buf->h, T * d, s) == cudaSuccess;
+  // Q, K, V as one GEMM when the caller laid them out for it: the three packed matrices and their
+  // betas back to back (one [3d, d] matrix with a beta per d rows) and q, k, v as the column
+  // blocks of one [T, 3d] buffer.
+  const size_t wbytes = (size_t)prefill_bytes(d, d);
+  const __half* qh = reinterpret_cast<const __half*>(buf->q);
+  const bool fused_qkv = ld_qkv == 3 * d && w->W_k == w->W_q + wbytes && w->W_v == w->W_k + wbytes &&
+                         w->beta_k == w->beta_q + 1 && w->beta_v == w->beta_k + 1 &&
+                         buf->k == (const void*)(qh + d) && buf->v == (const void*)(qh + 2 * d);
+  bool ok = quant(x, d, BL_ABSMAX);
+  if (fused_qkv) {
+    ok = ok && matmul(d, 3 * d, w->W_q, w->beta_q, d, buf->q, ld_qkv, false, nullptr);
+  } else {
+    ok = ok && matmul(d, d, w->W_q, w->beta_q, 0, buf->q, ld_qkv, false, nullptr)
+            && matmul(d, d, w->W_k, w->beta_k, 0, buf->k, ld_qkv, false, nullptr)
+            && matmul(d, d, w->W_v, w->beta_v, 0, buf->v, ld_qkv, false, nullptr);
+  }
+  ok = ok && launch_attention_causal(buf->q, buf->k, buf->v, buf->a, batch, seq, heads, ld_qkv, d, s) == cudaSuccess
+      && quant(buf->a, d, BL_ABSMAX) && matmul(d, d, w->W_o, w->beta_o, 0, buf->h, d, false, x)
+      && quant(buf->h, d, BL_ABSMAX) && matmul(d, ffn, w->W_up, w->beta_up, 0, buf->u, ffn, true, nullptr)
+      && quant(buf->u, ffn, BL_ETA) && matmul(ffn, d, w->W_down, w->beta_down, 0, y, d, false, buf->h);
   return ok ? BL_OK : BL_ERR_CUDA;
 }
 

@@ -126,6 +126,9 @@ __device__ __forceinline__ float dequant_term(int acc, float beta_g, float gamma
   return v;
 }
 
+__device__ __forceinline__ float in_cast(float v) { return v; }
+__device__ __forceinline__ float in_cast(__half v) { return __half2float(v); }
+__device__ __forceinline__ float in_cast(__nv_bfloat16 v) { return __bfloat162float(v); }
 template <typename T> __device__ __forceinline__ T out_cast(float f);
 template <> __device__ __forceinline__ float out_cast<float>(float f) { return f; }
 template <> __device__ __forceinline__ __half out_cast<__half>(float f) { return __float2half_rn(f); }
@@ -154,6 +157,12 @@ struct GemmArgs {
   void* y; bl_dtype yt;                            // dequantised output, or nullptr
   const float* beta; const float* gamma; const float* eta; bl_gran gran;
   const int32_t* rowsum; int eta_correction;
+  // Epilogue options of the dequantising kernels (all zero: Eq. 11 as is, dense y).
+  int64_t beta_rows;                               // output features per beta block (0: one block);
+                                                   // beta is [N/beta_rows, G], rowsum stays [N, G]
+  int relu;                                        // y = max(y, 0) before the residual
+  const void* residual; int64_t ld_res;            // y += residual[m, n] (dtype yt, row stride ld_res)
+  int64_t ld_y;                                    // row stride of y in elements (0: N)
   uint32_t* status;                                // device status word (tensor-core path)
   void* scratch;                                   // gemm_tc_scratch_bytes(G) bytes (tensor-core path)
 };

@@ -79,7 +79,8 @@ gemm_simple_kernel(GemmArgs a) {
           if (kDequant) {
             const int64_t sc = (a.gran == BL_PER_TOKEN) ? m * a.G + g : g;
             const bool corr = a.eta_correction != 0;
-            fsum[i][j] += dequant_term(acc[i][j], a.beta[g], a.gamma[sc], corr ? a.eta[sc] : 0.f,
+            const int64_t bb = a.beta_rows > 0 ? n / a.beta_rows : 0;
+            fsum[i][j] += dequant_term(acc[i][j], a.beta[bb * a.G + g], a.gamma[sc], corr ? a.eta[sc] : 0.f,
                                        corr ? a.rowsum[n * a.G + g] : 0, corr);
           } else {
             a.acc[((int64_t)g * a.M + m) * a.N + n] = acc[i][j];
@@ -97,7 +98,12 @@ gemm_simple_kernel(GemmArgs a) {
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int64_t n = n0 + tx * 4 + j;
-        if (m < a.M && n < a.N) y[m * a.N + n] = out_cast<TY>(fsum[i][j]);
+        if (m < a.M && n < a.N) {
+          float v = fsum[i][j];
+          if (a.relu) v = fmaxf(v, 0.f);
+          if (a.residual) v += in_cast(reinterpret_cast<const TY*>(a.residual)[m * a.ld_res + n]);
+          y[m * (a.ld_y > 0 ? a.ld_y : a.N) + n] = out_cast<TY>(v);
+        }
       }
     }
   }

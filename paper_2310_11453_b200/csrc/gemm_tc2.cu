@@ -316,12 +316,11 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
         got = __all_sync(0xFFFFFFFFu, got);
         if (!got) { ok = false; break; }
         tc_fence_after();
-        float scale = 0.f, eta_beta = 0.f;
+        float gamma_m = 0.f, eta_m = 0.f;
         if (kMode == 1 && m_ok) {
           const int64_t sc = (a.gran == BL_PER_TOKEN) ? m * a.G + g : g;
-          const float beta_g = a.beta[g];
-          scale = beta_g * a.gamma[sc] * kInvQb;
-          if (correct) eta_beta = a.eta[sc] * beta_g;
+          gamma_m = a.gamma[sc];
+          if (correct) eta_m = a.eta[sc];
         }
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * (uint32_t)kBN;
 #pragma unroll 1
@@ -343,6 +342,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
               }
             }
           } else {
+            // beta of this 32-column chunk (beta blocks are multiples of 32 output features)
+            const float beta_c = a.beta[(a.beta_rows > 0 ? n0 / a.beta_rows : 0) * a.G + g];
+            const float scale = beta_c * gamma_m * kInvQb, eta_beta = eta_m * beta_c;
             float v[32];
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
@@ -366,8 +368,29 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
               }
             }
             if (g + 1 == a.G && m_ok) {
-              TY* dst = reinterpret_cast<TY*>(a.y) + m * a.N + n0;
-              const bool vec_ok = (n0 + 32 <= a.N) && ((a.N * sizeof(TY)) % 16 == 0);
+              if (a.relu) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = fmaxf(v[i], 0.f);
+              }
+              if (a.residual) {
+                const TY* res = reinterpret_cast<const TY*>(a.residual) + m * a.ld_res + n0;
+                if (n0 + 32 <= a.N && (a.ld_res * sizeof(TY)) % 16 == 0) {
+                  constexpr int kPer = 16 / (int)sizeof(TY);           // elements per 16-byte load
+#pragma unroll
+                  for (int i = 0; i < 32 / kPer; ++i) {
+                    const uint4 w = *reinterpret_cast<const uint4*>(res + i * kPer);
+                    const TY* e = reinterpret_cast<const TY*>(&w);
+#pragma unroll
+                    for (int j = 0; j < kPer; ++j) v[i * kPer + j] += in_cast(e[j]);
+                  }
+                } else {
+#pragma unroll
+                  for (int i = 0; i < 32; ++i) if (n0 + i < a.N) v[i] += in_cast(res[i]);
+                }
+              }
+              const int64_t ldy = a.ld_y > 0 ? a.ld_y : a.N;
+              TY* dst = reinterpret_cast<TY*>(a.y) + m * ldy + n0;
+              const bool vec_ok = (n0 + 32 <= a.N) && ((ldy * sizeof(TY)) % 16 == 0);
               store_row32<TY>(dst, v, n0, a.N, vec_ok);
             }
           }

@@ -8,7 +8,9 @@ intermediate buffers):
   * each BitLinear: int8 codes within +-1 on <= 1e-4 of the elements; sampled outputs within 1e-3 of
     the output RMS of the oracle's Eq. 11 on the GPU's own codes, plus the fp16 rounding of the store;
   * attention: sampled rows against the fp64 definition within fp16 tolerance;
-  * residual adds and ReLU: bit-exact against the same fp16 operation on the CPU."""
+  * residual adds and ReLU (run in the GEMM epilogues): bit-exact against the fp32 projection with
+    the same operation applied and one rounding to fp16;
+  * Q, K, V as one [3d, d] GEMM and as three GEMMs write the same bits."""
 import numpy as np
 import pytest
 import torch
@@ -54,50 +56,57 @@ def check_bitlinear_stage(x_in, y_out, w_ref, mode, samples, seed):
     assert (np.abs(y_gpu - y_stage) <= 1e-3 * rms + np.abs(y_stage) * 2.0 ** -11 + 1e-7).all()
 
 
-def run_block(batch, seq, heads, ffn, seed, attn_rows):
+def run_block(batch, seq, heads, ffn, seed, attn_rows, fused_qkv):
     d = heads * 128
     T = batch * seq
     x = synth.make_x(T, d, torch.float16, seed=seed, outliers=False).to(DEV)
     w_ref, w_gpu = make_block(d, ffn, seed)
-    out = B.block_forward(x, w_gpu, batch, seq, heads, ffn)
+    if fused_qkv:
+        w_gpu = B.fuse_qkv_weights(w_gpu)
+    out = B.block_forward(x, w_gpu, batch, seq, heads, ffn, fused_qkv=fused_qkv)
     assert B.ws_status(out["ws"]) == B.OK
+
+    def proj32(src, name, N, mode=B.ABSMAX):
+        return B.forward(src, w_gpu[name]["W_packed"], w_gpu[name]["beta"], N, mode=mode, gran=B.PER_TOKEN,
+                         layout=B.PREFILL, out_dtype=torch.float32)
     # stages that write their BitLinear output straight to an inspectable buffer
     for name, src, dst in (("q", x, out["q"]), ("k", x, out["k"]), ("v", x, out["v"])):
         check_bitlinear_stage(src, dst, w_ref[name], "absmax", 2000, seed)
     # attention core on the GPU's q, k, v
     rows = np.unique(np.concatenate([[0, 1, 63, 64, seq - 1, T - seq, T - 1],
                                      np.random.default_rng(seed).integers(0, T, attn_rows)])).astype(np.int64)
-    a_ref = O.attention_rows(as_f32_np(out["q"]), as_f32_np(out["k"]), as_f32_np(out["v"]), batch, seq, heads, 128, rows)
+    a_ref = O.attention_rows(as_f32_np(out["q"].contiguous()), as_f32_np(out["k"].contiguous()),
+                             as_f32_np(out["v"].contiguous()), batch, seq, heads, 128, rows)
     a_gpu = out["a"].cpu().float().numpy()[rows].astype(np.float64)
     scale = np.abs(a_ref).max()
     assert np.abs(a_gpu - a_ref).max() <= 4e-3 * scale          # fp16 probabilities and outputs
     assert np.sqrt(((a_gpu - a_ref) ** 2).mean()) <= 1e-3 * scale
     # O projection + residual: h = x + BitLinear_O(a); recompute the projection alone for the stage check
-    o_proj = B.forward(out["a"], w_gpu["o"]["W_packed"], w_gpu["o"]["beta"], d, gran=B.PER_TOKEN, layout=B.PREFILL,
-                       out_dtype=torch.float16)
-    check_bitlinear_stage(out["a"], o_proj, w_ref["o"], "absmax", 2000, seed + 1)
-    assert torch.equal(out["h"], o_proj + x)                        # fp16 add, bit for bit
+    o_proj = proj32(out["a"], "o", d)
+    check_bitlinear_stage(out["a"], o_proj.half(), w_ref["o"], "absmax", 2000, seed + 1)
+    assert torch.equal(out["h"], (o_proj + x.float()).half())       # fp32 add, one rounding, bit for bit
     # up projection + ReLU
-    up = B.forward(out["h"], w_gpu["up"]["W_packed"], w_gpu["up"]["beta"], ffn, gran=B.PER_TOKEN, layout=B.PREFILL,
-                   out_dtype=torch.float16)
-    check_bitlinear_stage(out["h"], up, w_ref["up"], "absmax", 2000, seed + 2)
-    assert torch.equal(out["u"], torch.relu(up))
+    up = proj32(out["h"], "up", ffn)
+    check_bitlinear_stage(out["h"], up.half(), w_ref["up"], "absmax", 2000, seed + 2)
+    assert torch.equal(out["u"], torch.relu(up).half())
     # down projection (eta form on the ReLU output) + residual
-    down = B.forward(out["u"], w_gpu["down"]["W_packed"], w_gpu["down"]["beta"], d, mode=B.ETA, gran=B.PER_TOKEN,
-                     layout=B.PREFILL, out_dtype=torch.float16)
-    check_bitlinear_stage(out["u"], down, w_ref["down"], "eta", 2000, seed + 3)
-    assert torch.equal(out["y"], down + out["h"])
+    down = proj32(out["u"], "down", d, mode=B.ETA)
+    check_bitlinear_stage(out["u"], down.half(), w_ref["down"], "eta", 2000, seed + 3)
+    assert torch.equal(out["y"], (down + out["h"].float()).half())
     assert torch.isfinite(out["y"]).all()
     return out
 
 
 def test_block_small():
-    run_block(batch=2, seq=128, heads=2, ffn=1024, seed=50, attn_rows=64)
+    a = run_block(batch=2, seq=128, heads=2, ffn=1024, seed=50, attn_rows=64, fused_qkv=False)
+    b = run_block(batch=2, seq=128, heads=2, ffn=1024, seed=50, attn_rows=64, fused_qkv=True)
+    for name in ("q", "k", "v", "a", "h", "u", "y"):
+        assert torch.equal(a[name], b[name]), name
 
 
 def test_block_config4_full_size():
-    # d = 2048, 16 heads, FFN 8192, batch 4 x seq 2048
-    run_block(batch=4, seq=2048, heads=16, ffn=8192, seed=60, attn_rows=48)
+    # d = 2048, 16 heads, FFN 8192, batch 4 x seq 2048, in the layout the benchmark times
+    run_block(batch=4, seq=2048, heads=16, ffn=8192, seed=60, attn_rows=48, fused_qkv=True)
 
 
 def test_attention_alone_against_definition():

@@ -439,3 +439,41 @@ def test_attention_closed_forms():
     o3 = O.attention_rows(q3, k, v, B, S, H, D, np.array([10]))
     scores = (q3[10, :D].astype(np.float64) @ k[:11, :D].astype(np.float64).T) / np.sqrt(D)
     assert np.abs(o3[0, :D] - v[int(np.argmax(scores)), :D]).max() < 1e-6
+
+
+# ---------------------------------------------------------------- N-split groups (Eq. 13 along N)
+
+def test_binarize_nsplit_blocks_have_their_own_alpha_and_beta():
+    rng = np.random.default_rng(7)
+    N, K, NB, G = 24, 64, 3, 2
+    # blocks with clearly different means and spreads
+    W = np.concatenate([rng.normal(m, s, size=(N // NB, K)) for m, s in ((0.5, 0.1), (-0.2, 1.0), (0.0, 0.01))])
+    W = W.astype(np.float32)
+    r = O.binarize_nsplit(W, NB, G=G)
+    rows, Kg = N // NB, K // G
+    for j in range(NB):
+        for g in range(G):
+            blk = W[j * rows:(j + 1) * rows, g * Kg:(g + 1) * Kg].astype(np.float64)
+            assert abs(r["alpha"][j, g] - blk.mean()) < 1e-12
+            assert abs(r["beta"][j, g] - np.abs(blk).mean()) < 1e-12
+            want = (blk > blk.mean())
+            got = np.unpackbits(r["bits"][j * rows:(j + 1) * rows], axis=1, bitorder="little")[:, g * Kg:(g + 1) * Kg]
+            assert np.array_equal(got.astype(bool), want)
+    # one block is the plain per-matrix binarisation
+    one = O.binarize_nsplit(W, 1, G=G)
+    ref = O.binarize(W, G=G)
+    assert np.array_equal(one["bits"], ref["bits"]) and np.array_equal(one["alpha"][0], ref["alpha"])
+
+
+def test_dequant_nsplit_scales_each_block_by_its_beta():
+    rng = np.random.default_rng(8)
+    G, M, N, NB = 2, 5, 12, 3
+    acc = rng.integers(-1000, 1000, size=(G, M, N)).astype(np.int32)
+    beta = rng.uniform(0.1, 2.0, size=(NB, G))
+    gamma = rng.uniform(1.0, 5.0, size=(M, G))
+    y = O.dequant_nsplit(acc, beta, gamma, gran=O.PER_TOKEN)
+    want = np.zeros((M, N))
+    for m in range(M):
+        for n in range(N):
+            want[m, n] = sum(acc[g, m, n] * beta[n // (N // NB), g] * gamma[m, g] / 128.0 for g in range(G))
+    assert np.allclose(y, want, rtol=1e-13, atol=0)
