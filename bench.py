@@ -348,6 +348,37 @@ def bench_decode(B, synth, dev, peaks):
     bytes_per_call = N * K / 8 + 2 * K + 2 * N
     gbs = bytes_per_call / (out["hbm"] * 1e-6) / 1e9
 
+    # small batches through bitlinear_gemv_decode_batch: M tokens share one pass over the weights
+    batch = {}
+    bcalls = 400
+    yb = torch.empty((16, N), dtype=torch.float16, device=dev)
+    for Mb in (1, 2, 4, 8, 16):
+        def issue_batch():
+            for i in range(bcalls):
+                p = packs[i % nbuf]
+                r0 = (i * Mb) % (calls - Mb)
+                B.gemv_decode_batch(x[r0:r0 + Mb], p["W_packed"], p["beta"], N, y=yb[:Mb])
+        issue_batch()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            issue_batch()
+        for _ in range(2):
+            graph.replay()
+        torch.cuda.synchronize()
+        times = []
+        for _ in range(5):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            graph.replay()
+            b.record()
+            torch.cuda.synchronize()
+            times.append(a.elapsed_time(b))
+        us = statistics.median(times) / bcalls * 1e3
+        batch[f"M{Mb}"] = {"us_per_call": us, "us_per_token": us / Mb,
+                           "weight_gbs": (N * K / 8 + Mb * 2 * (K + N)) / (us * 1e-6) / 1e9}
+        del graph
+
     def rate(us):
         return bytes_per_call / (us * 1e-6) / 1e9
 
@@ -356,6 +387,9 @@ def bench_decode(B, synth, dev, peaks):
                         "(every call ordered after the one before it)",
             "us_per_call": out["hbm"], "us_per_call_l2_hot": out["l2_hot"], "bytes_per_call": bytes_per_call,
             "gpu_launches": calls,
+            "small_batch": {"note": "bitlinear_gemv_decode_batch, M tokens per call (one launch per 8 tokens), "
+                                    "400 calls in one CUDA graph over the same 64 weight buffers, one stream",
+                            **batch},
             "independent_streams": {
                 "note": "same 1000 calls spread round-robin over 2 / 4 streams inside the graph: calls on "
                         "different streams do not wait for one another",

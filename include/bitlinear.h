@@ -226,6 +226,19 @@ bl_status bitlinear_gemv_decode(const void* x, bl_dtype xt, int64_t K, int64_t N
                                 const uint8_t* W_packed, const float* beta,
                                 const int32_t* rowsum, void* y, bl_dtype yt, void* stream);
 
+/* bitlinear_gemv_decode for a small batch: M tokens (decode with a few sequences in flight, the
+ * per-token inference of Sec. 2.1 with one weight stream shared by the batch).  Each token gets
+ * its own LN statistics, gamma and eta (Eq. 12, 4-6 per token); up to 8 tokens share one pass
+ * over the packed weights (tensor-core mma on bit planes of the packed words), larger M runs
+ * ceil(M/8) passes with the weights served from L2.
+ *   x [M,K] of dtype xt;  y [M,N] of dtype yt;  W_packed in DECODE layout.
+ *   K % 256 == 0, (K/G) % 256 == 0, N % 16 == 0, min(M, 8) * (K + 16) <= 155 KB (BL_ERR_SHAPE otherwise).
+ * No workspace, no device-side waits. */
+bl_status bitlinear_gemv_decode_batch(const void* x, bl_dtype xt, int64_t M, int64_t K, int64_t N, int G,
+                                      int b, bl_quant_mode mode, float ln_eps, int eta_correction,
+                                      const uint8_t* W_packed, const float* beta, const int32_t* rowsum,
+                                      void* y, bl_dtype yt, void* stream);
+
 /* Causal self-attention core of the decoder block (Sec. 2, Fig. 2b; the paper keeps it in high
  * precision): per batch and head O = softmax(Q K^T / sqrt(d_h) + causal mask) V, fp16 in and out,
  * fp32 softmax statistics and accumulators.  No positional encoding.

@@ -28,7 +28,7 @@ EXPORTS = [
     "bitlinear_layout_index", "bitlinear_binarize_pack", "bitlinear_quant_act", "bitlinear_quant_act_noalloc",
     "bitlinear_forward", "bitlinear_matmul_i32", "bitlinear_matmul_dequant", "bitlinear_gemv_decode",
     "bitlinear_attention_causal", "bitlinear_block_forward", "bitlinear_ws_status",
-    "bitlinear_matmul_dequant_ex", "bitlinear_binarize_pack_nsplit",
+    "bitlinear_matmul_dequant_ex", "bitlinear_binarize_pack_nsplit", "bitlinear_gemv_decode_batch",
 ]
 
 _DTYPES = {torch.float32: F32, torch.float16: F16, torch.bfloat16: BF16}
@@ -84,6 +84,9 @@ def lib():
         L.bitlinear_matmul_dequant_ex.restype = ci
         L.bitlinear_matmul_dequant_ex.argtypes = [vp, i64, i64, i64, ci, ci, vp, vp, ci, vp, ci, vp, vp, vp, vp, ci,
                                                   vp, sz, vp]
+        L.bitlinear_gemv_decode_batch.restype = ci
+        L.bitlinear_gemv_decode_batch.argtypes = [vp, ci, i64, i64, i64, ci, ci, ci, C.c_float, ci, vp, vp, vp, vp,
+                                                  ci, vp]
         L.bitlinear_binarize_pack_nsplit.restype = ci
         L.bitlinear_binarize_pack_nsplit.argtypes = [vp, ci, i64, i64, ci, ci, ci, vp, vp, vp, vp, vp, vp, sz, vp]
         _lib = L
@@ -289,6 +292,19 @@ def gemv_decode(x, W_packed, beta, N, G=1, mode=ABSMAX, ln_eps=1e-5, rowsum=None
                                        1 if eta_correction else 0, _ptr(W_packed), _ptr(beta),
                                        _ptr(rowsum), _ptr(y), _dt(y), _stream())
     _check(code, "bitlinear_gemv_decode")
+    return y
+
+
+def gemv_decode_batch(x, W_packed, beta, N, G=1, mode=ABSMAX, ln_eps=1e-5, rowsum=None,
+                      eta_correction=False, out_dtype=None, b=8, y=None):
+    """bitlinear_gemv_decode_batch.  x [M,K]; W_packed in DECODE layout; returns y [M,N]."""
+    M, K = x.shape
+    if y is None:
+        y = torch.empty((M, N), dtype=out_dtype or x.dtype, device=x.device)
+    code = lib().bitlinear_gemv_decode_batch(_ptr(x), _dt(x), M, K, N, G, b, mode, float(ln_eps),
+                                             1 if eta_correction else 0, _ptr(W_packed), _ptr(beta),
+                                             _ptr(rowsum), _ptr(y), _dt(y), _stream())
+    _check(code, "bitlinear_gemv_decode_batch")
     return y
 
 

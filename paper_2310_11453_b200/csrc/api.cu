@@ -307,6 +307,24 @@ bl_status bitlinear_gemv_decode(const void* x, bl_dtype xt, int64_t K, int64_t N
   return launch_gemv_decode(a, (cudaStream_t)stream) == cudaSuccess ? BL_OK : BL_ERR_CUDA;
 }
 
+bl_status bitlinear_gemv_decode_batch(const void* x, bl_dtype xt, int64_t M, int64_t K, int64_t N, int G,
+                                      int b, bl_quant_mode mode, float ln_eps, int eta_correction,
+                                      const uint8_t* W_packed, const float* beta, const int32_t* rowsum,
+                                      void* y, bl_dtype yt, void* stream) {
+  if (!x || !W_packed || !beta || !y) return BL_ERR_NULL;
+  if (eta_correction && !rowsum) return BL_ERR_NULL;
+  if (M <= 0 || N <= 0) return BL_ERR_SHAPE;
+  bl_status st = check_kg(K, G);
+  if (st != BL_OK) return st;
+  if (b != 8 || !valid_dtype(xt) || !valid_dtype(yt)) return BL_ERR_UNSUPPORTED;
+  if (mode != BL_ABSMAX && mode != BL_ETA) return BL_ERR_UNSUPPORTED;
+  if (eta_correction && mode != BL_ETA) return BL_ERR_UNSUPPORTED;
+  if (!gemv_batch_supported(M, K, N, G)) return BL_ERR_SHAPE;
+  if (!aligned16(x) || !aligned16(W_packed) || !aligned16(y)) return BL_ERR_ALIGN;
+  GemvArgs a{x, xt, K, N, G, mode, ln_eps, eta_correction ? 1 : 0, W_packed, beta, rowsum, y, yt};
+  return launch_gemv_batch(a, M, (cudaStream_t)stream) == cudaSuccess ? BL_OK : BL_ERR_CUDA;
+}
+
 bl_status bitlinear_attention_causal(const void* q, const void* k, const void* v, void* o, int batch, int seq,
                                      int heads, int head_dim, int64_t ld, int64_t ld_o, void* stream) {
   if (!q || !k || !v || !o) return BL_ERR_NULL;

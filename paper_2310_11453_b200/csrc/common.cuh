@@ -178,6 +178,9 @@ struct GemvArgs {
   void* y; bl_dtype yt;
 };
 cudaError_t launch_gemv_decode(const GemvArgs& a, cudaStream_t s);
+// The same for M tokens (x [M,K], y [M,N]) sharing one pass over the weights per 8 tokens.
+cudaError_t launch_gemv_batch(const GemvArgs& a, int64_t M, cudaStream_t s);
+bool gemv_batch_supported(int64_t M, int64_t K, int64_t N, int G);
 
 // Decoder-block glue (fp16): causal attention core and the elementwise steps.
 cudaError_t launch_attention_causal(const void* q, const void* k, const void* v, void* o, int batch, int S,

@@ -1,0 +1,83 @@
+"""Small-batch decode (M tokens sharing one pass over the DECODE-packed weights) against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2310_11453_b200 import binding as B
+from paper_2310_11453_b200 import synth
+from tests.util import as_f32_np
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+DT = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}
+
+
+@pytest.mark.parametrize("M,K,N,G,dtype,mode,relu", [
+    (8, 4096, 16384, 1, "f16", "absmax", False),     # config c2's layer with a full batch of 8
+    (1, 256, 16, 1, "f32", "absmax", False),         # smallest shape, one token
+    (3, 1024, 48, 2, "bf16", "eta", True),           # groups along K, eta form
+    (13, 2048, 160, 1, "f16", "absmax", False),      # two launches, ragged second batch of 5
+    (5, 8192, 64, 1, "bf16", "absmax", False),       # K above two register batches of weights
+    (2, 7168, 112, 7, "bf16", "eta", True),          # seven groups of 1024
+])
+def test_gemv_decode_batch(M, K, N, G, dtype, mode, relu):
+    x = synth.make_x(M, K, DT[dtype], seed=K + N + M, outliers=False, relu=relu)
+    W = synth.make_w(N, K, torch.float32, seed=K)
+    omode = O.ETA if mode == "eta" else O.ABSMAX
+    w_ref = O.binarize(W.numpy(), G=G)
+    w_gpu = B.binarize_pack(W.to(DEV), G=G, layout=B.DECODE)
+    xd = x.to(DEV)
+    # the kernel's LN + Quant is the per-token path of bitlinear_quant_act: same codes, gamma, eta
+    q = B.quant_act(xd, G=G, mode=omode, gran=B.PER_TOKEN, ln_eps=1e-5)
+    ref_q = O.quant_act(as_f32_np(x), G=G, mode=omode, gran=O.PER_TOKEN, ln_eps=1e-5)
+    codes = q["x_q"].cpu().numpy()
+    diff = codes.astype(np.int32) - ref_q["codes"].astype(np.int32)
+    assert np.abs(diff).max() <= 1 and np.count_nonzero(diff) <= max(4, 2e-4 * diff.size)
+    acc = O.matmul(codes, w_ref["bits"], G=G)
+    for corr in ([False, True] if mode == "eta" else [False]):
+        y = B.gemv_decode_batch(xd, w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode, ln_eps=1e-5,
+                                rowsum=w_gpu["rowsum"], eta_correction=corr, out_dtype=torch.float32)
+        torch.cuda.synchronize()
+        want = O.dequant(acc, w_gpu["beta"].cpu().numpy().astype(np.float64),
+                         q["gamma"].cpu().numpy().astype(np.float64), gran=O.PER_TOKEN,
+                         eta=q["eta"].cpu().numpy().astype(np.float64), rowsum=w_ref["rowsum"], eta_correction=corr)
+        rms = np.sqrt((want ** 2).mean())
+        assert np.abs(y.cpu().numpy().astype(np.float64) - want).max() <= 1e-3 * rms
+    # 16-bit output is the rounding of the fp32 one
+    y32 = B.gemv_decode_batch(xd, w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode, out_dtype=torch.float32)
+    if dtype != "f32":
+        y16 = B.gemv_decode_batch(xd, w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode, out_dtype=DT[dtype])
+        assert torch.equal(y16, y32.to(DT[dtype]))
+    # a token's result does not depend on what else is in the batch
+    if M > 1:
+        y_one = B.gemv_decode_batch(xd[M - 1:M].contiguous(), w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode,
+                                    out_dtype=torch.float32)
+        assert torch.equal(y_one[0], y32[M - 1])
+
+
+def test_gemv_decode_batch_integer_definition_exactly():
+    # LN skipped and gamma planted at 128 (an element equal to 128 in every token): the codes are
+    # the inputs themselves, so y must equal acc * beta as computed by the oracle's integer matmul.
+    M, K, N = 6, 1024, 96
+    codes = synth.make_codes(M, K, seed=9)
+    x = codes.to(torch.float32)
+    x[:, 0] = 128.0                                                  # gamma = 128, its code clips to 127
+    W = synth.make_w(N, K, torch.float32, seed=9)
+    w_ref = O.binarize(W.numpy())
+    w_gpu = B.binarize_pack(W.to(DEV), layout=B.DECODE)
+    y = B.gemv_decode_batch(x.to(DEV), w_gpu["W_packed"], w_gpu["beta"], N, ln_eps=-1.0, out_dtype=torch.float32)
+    c = codes.numpy().copy()
+    c[:, 0] = 127
+    acc = O.matmul(c, w_ref["bits"])[0].astype(np.float64)
+    want = (acc * float(w_gpu["beta"][0])).astype(np.float32)
+    assert np.allclose(y.cpu().numpy(), want, rtol=3e-7, atol=0)
+
+
+def test_gemv_decode_batch_argument_checks():
+    x = torch.zeros((2, 384), dtype=torch.float16, device=DEV)
+    w = torch.zeros(64, dtype=torch.uint8, device=DEV)
+    beta = torch.ones(1, device=DEV)
+    with pytest.raises(B.BitLinearError) as e:                      # K not a multiple of 256
+        B.gemv_decode_batch(x, w, beta, 16)
+    assert e.value.code == B.ERR_SHAPE
