@@ -143,7 +143,8 @@ struct StepIter {
   __device__ bool last() const { return t + 1 == spg; }
 };
 
-// kMode 0: write int32 accumulators acc[g,m,n].  kMode 1: write y (Eq. 11).
+// kMode 0: write int32 accumulators acc[g,m,n].  kMode 1: write y (Eq. 11).  kMode 2: the same with
+// the epilogue options (beta per block of output features, ReLU, residual, row stride of y).
 template <int kMode, typename TY>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_bytes) {
@@ -305,7 +306,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
     uint32_t pass = 0;
     bool ok = true;
     float* run = reinterpret_cast<float*>(reinterpret_cast<char*>(a.scratch) + (size_t)blockIdx.x * kScratchPerCta);
-    const bool correct = (kMode == 1) && a.eta_correction != 0;
+    const bool correct = (kMode >= 1) && a.eta_correction != 0;
     for (PairIter it(tiles, m_tiles); ok && it.valid(); it.next()) {
       const int64_t m = (int64_t)it.m_tile() * kPairM + rank * kBM + row;
       const int64_t n_base = (int64_t)it.n_tile() * kBN;
@@ -316,18 +317,23 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
         got = __all_sync(0xFFFFFFFFu, got);
         if (!got) { ok = false; break; }
         tc_fence_after();
-        float gamma_m = 0.f, eta_m = 0.f;
-        if (kMode == 1 && m_ok) {
+        // one beta for the tile (beta_rows == 0) or one per 32-column chunk, loaded below
+        float gamma_m = 0.f, eta_m = 0.f, beta_c = 0.f;
+        if (kMode >= 1 && m_ok) {
           const int64_t sc = (a.gran == BL_PER_TOKEN) ? m * a.G + g : g;
           gamma_m = a.gamma[sc];
           if (correct) eta_m = a.eta[sc];
         }
+        if (kMode == 1 || (kMode == 2 && a.beta_rows == 0)) beta_c = a.beta[g];
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * (uint32_t)kBN;
 #pragma unroll 1
         for (int c = 0; c < kBN / 32; ++c) {
+          const int64_t n0 = n_base + c * 32;
+          // beta blocks are multiples of 32 output features: one value per chunk, fetched while the
+          // accumulators travel from tensor memory
+          if (kMode == 2 && a.beta_rows > 0 && n0 < a.N) beta_c = __ldg(a.beta + (n0 / a.beta_rows) * a.G + g);
           uint32_t r[32];
           tmem_ld32(taddr + (uint32_t)(c * 32), r);
-          const int64_t n0 = n_base + c * 32;
           if (n0 >= a.N) continue;                           // uniform across the warp
           if (kMode == 0) {
             if (m_ok) {
@@ -342,8 +348,6 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
               }
             }
           } else {
-            // beta of this 32-column chunk (beta blocks are multiples of 32 output features)
-            const float beta_c = a.beta[(a.beta_rows > 0 ? n0 / a.beta_rows : 0) * a.G + g];
             const float scale = beta_c * gamma_m * kInvQb, eta_beta = eta_m * beta_c;
             float v[32];
 #pragma unroll
@@ -368,11 +372,11 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
               }
             }
             if (g + 1 == a.G && m_ok) {
-              if (a.relu) {
+              if (kMode == 2 && a.relu) {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) v[i] = fmaxf(v[i], 0.f);
               }
-              if (a.residual) {
+              if (kMode == 2 && a.residual) {
                 const TY* res = reinterpret_cast<const TY*>(a.residual) + m * a.ld_res + n0;
                 if (n0 + 32 <= a.N && (a.ld_res * sizeof(TY)) % 16 == 0) {
                   constexpr int kPer = 16 / (int)sizeof(TY);           // elements per 16-byte load
@@ -388,7 +392,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
                   for (int i = 0; i < 32; ++i) if (n0 + i < a.N) v[i] += in_cast(res[i]);
                 }
               }
-              const int64_t ldy = a.ld_y > 0 ? a.ld_y : a.N;
+              const int64_t ldy = (kMode == 2 && a.ld_y > 0) ? a.ld_y : a.N;
               TY* dst = reinterpret_cast<TY*>(a.y) + m * ldy + n0;
               const bool vec_ok = (n0 + 32 <= a.N) && ((ldy * sizeof(TY)) % 16 == 0);
               store_row32<TY>(dst, v, n0, a.N, vec_ok);
@@ -427,7 +431,7 @@ cudaError_t launch(const GemmArgs& a, cudaStream_t s) {
           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return cudaErrorInvalidValue;
-  static bool attr_set[2][3] = {};
+  static bool attr_set[3][3] = {};
   auto kern = gemm_tc2_kernel<kMode, TY>;
   const int ti = kMode == 0 ? 0 : (int)a.yt;
   if (!attr_set[kMode][ti]) {
@@ -443,7 +447,7 @@ cudaError_t launch(const GemmArgs& a, cudaStream_t s) {
   int64_t clusters = (sms < kMaxCtas ? sms : kMaxCtas) / 2;
   {
     // persistent grid: no more clusters than can be resident at once
-    static int resident[2][3] = {};
+    static int resident[3][3] = {};
     if (resident[kMode][ti] == 0) {
       cudaLaunchConfig_t cfg = {};
       cfg.gridDim = dim3((unsigned)(2 * clusters));
@@ -467,10 +471,11 @@ cudaError_t launch(const GemmArgs& a, cudaStream_t s) {
 
 cudaError_t launch_gemm_tc2(const GemmArgs& a, cudaStream_t s) {
   if (a.y == nullptr) return launch<0, float>(a, s);
+  const bool ext = a.beta_rows > 0 || a.relu || a.residual != nullptr || (a.ld_y > 0 && a.ld_y != a.N);
   switch (a.yt) {
-    case BL_F32: return launch<1, float>(a, s);
-    case BL_F16: return launch<1, __half>(a, s);
-    case BL_BF16: return launch<1, __nv_bfloat16>(a, s);
+    case BL_F32: return ext ? launch<2, float>(a, s) : launch<1, float>(a, s);
+    case BL_F16: return ext ? launch<2, __half>(a, s) : launch<1, __half>(a, s);
+    case BL_BF16: return ext ? launch<2, __nv_bfloat16>(a, s) : launch<1, __nv_bfloat16>(a, s);
   }
   return cudaErrorInvalidValue;
 }
