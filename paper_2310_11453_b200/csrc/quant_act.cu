@@ -2,9 +2,10 @@
 // quantisation (Eq. 4-6, 14).  HBM-bound: x is read once (per token) or twice (per tensor) with
 // 128-bit loads; the normalised row is never written to HBM.
 //
-// Two implementations.  Segments of up to 4096 16-bit (2048 fp32) features take the fast path in
-// the second half of this file: one warp per segment, the segment in registers.  Longer segments
-// take one CTA per (token m, group g) segment, staged in shared memory as fp32:
+// Two implementations.  Segments of up to 16 KB (8192 16-bit, 4096 fp32 features) that are a
+// multiple of 256 features take the fast path in the second half of this file: one warp per
+// segment, staged in shared memory.  Other segments take one CTA per (token m, group g) segment,
+// staged in shared memory as fp32:
 //   moments  sum, raw min/max, then sum of squared deviations      (quant_core.cuh)
 //   codes    one FMA + round per element, 8 codes per 8-byte store
 // Per-tensor scope splits in two kernels: the first leaves each segment's moments in the
@@ -136,13 +137,15 @@ tensor_codes(const T* __restrict__ x, int64_t K, int G, int mode, const TensorSc
 // ================================================================================================
 // Fast path: one warp per (token, group) segment, the segment staged in shared memory.
 //
-// Used when a segment is a whole number of 256-element pieces and at most 8 KB (K_g <= 4096 for
-// 16-bit inputs, <= 2048 for fp32), which covers every shape of the paper's model table.  The
+// Used when a segment is a whole number of 256-element pieces and at most 16 KB, which covers
+// every hidden size of the paper's model table and the FFN width up to the 1.3B model.  The
 // kernels are persistent: one CTA per SM; CTA c owns the contiguous segment range
 // [c*S/grid, (c+1)*S/grid) and its warps draw segments from it through a shared counter.  Each warp
-// has two 8 KB slots of shared memory: while it works on one, the asynchronous copies (cp.async,
-// 16 bytes per lane and instruction) of its next segment land in the other, so every warp keeps a
-// segment's worth of HBM traffic outstanding whatever it is computing.  Waiting is
+// has 16 KB of shared memory.  For segments of up to 8 KB these are two slots: while the warp works
+// on one, the asynchronous copies (cp.async, 16 bytes per lane and instruction) of its next
+// segment land in the other, so every warp keeps a segment's worth of HBM traffic outstanding
+// whatever it is computing.  A longer segment takes the whole area; its successor is copied after
+// the work on it, and the other eleven warps keep the memory system busy meanwhile.  Waiting is
 // cp.async.wait_group: no barrier objects, no spin loops.  A warp walks its segment in chunks of
 // 8 elements per lane (a short rolled loop: small code, few registers), with warp shuffles for
 // the reductions and no block barrier inside the loop.  Sums are fp32 inside a lane and fp64
@@ -154,7 +157,7 @@ constexpr int kSlotBytes = 8192;
 constexpr int kRowStage = kRowWarps * 2 * kSlotBytes;
 template <typename T> struct RowTraits {                      // chunk = 8 consecutive elements
   static constexpr int kVecPerChunk = sizeof(T) == 4 ? 2 : 1; // 16-byte pieces per chunk
-  static constexpr int kMaxKg = kSlotBytes / (int)sizeof(T);
+  static constexpr int kMaxKg = 2 * kSlotBytes / (int)sizeof(T);   // a warp's whole staging area
 };
 
 // ---- segment ranges and staging --------------------------------------------------------------------
@@ -213,16 +216,26 @@ __device__ __forceinline__ void for_each_segment(const T* __restrict__ x, int64_
   const int lane = threadIdx.x & 31;
   uint4* slots = reinterpret_cast<uint4*>(stage + (size_t)(threadIdx.x >> 5) * 2 * kSlotBytes);
   const RowRange rg = cta_range(segments);
+  // A segment of up to kSlotBytes leaves room for two slots (the next copy overlaps this body); a
+  // longer one (up to 2 * kSlotBytes) fills the warp's whole area and its successor is copied after
+  // the body, the other warps' copies and bodies covering for it.
+  const bool two_slots = Kg * (int)sizeof(T) <= kSlotBytes;
   int cur = 0;
   int64_t seg = first_seg;
   while (seg >= 0) {
-    const int64_t next =
-        stage_next<T>(x, rg, K, G, Kg, reverse, policy, counter, slots + (cur ^ 1) * (kSlotBytes / 16), lane);
-    cp_async_wait_but_newest();
+    int64_t next = -1;
+    if (two_slots) {
+      next = stage_next<T>(x, rg, K, G, Kg, reverse, policy, counter, slots + (cur ^ 1) * (kSlotBytes / 16), lane);
+      cp_async_wait_but_newest();
+    } else {
+      asm volatile("cp.async.wait_all;" ::: "memory");
+    }
     __syncwarp();
     body(seg, slots + cur * (kSlotBytes / 16));
     __syncwarp();                                    // every lane is done with the slot before it is refilled
-    seg = next; cur ^= 1;
+    if (two_slots) cur ^= 1;
+    else next = stage_next<T>(x, rg, K, G, Kg, reverse, policy, counter, slots, lane);
+    seg = next;
   }
 }
 // First draw of a warp (into slot 0), split off so that a kernel can put work between it and the loop.

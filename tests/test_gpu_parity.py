@@ -136,10 +136,13 @@ QUANT_CASES = [
     (17, 28672, 8, "bf16", "eta", "tensor", False, True),    # c5-shaped rows
     (17, 28672, 8, "bf16", "absmax", "token", True, False),
     (5, 8, 1, "f32", "absmax", "token", False, False),
-    (9, 8192, 1, "bf16", "absmax", "token", True, False),    # longer than a warp's registers: CTA path
+    (9, 8192, 1, "bf16", "absmax", "token", True, False),    # 16 KB segments: one slot per warp
     (9, 8192, 1, "f16", "eta", "tensor", False, True),
     (7, 4096, 1, "f32", "absmax", "tensor", True, False),
-    (3, 2048, 1, "f32", "eta", "token", False, True),        # the longest fp32 segment of the warp path
+    (3, 2048, 1, "f32", "eta", "token", False, True),        # the longest fp32 segment with two slots per warp
+    (40, 8192, 1, "f16", "eta", "token", False, True),       # more 16 KB segments than warps in a CTA
+    (5, 16384, 1, "bf16", "absmax", "token", True, False),   # longer than a warp's staging area: CTA path
+    (5, 16384, 1, "bf16", "eta", "tensor", False, True),
 ]
 
 
