@@ -287,9 +287,11 @@ rows_tensor_stats(const T* __restrict__ x, int64_t segments, int64_t K, int G, i
   const int lane = threadIdx.x & 31;
   if (threadIdx.x == 0) counter = 0;
   if (threadIdx.x < BL_MAX_GROUPS) { part_lo[threadIdx.x] = ~0ull; part_hi[threadIdx.x] = 0ull; }
-  pdl_launch_dependents();
   __syncthreads();
   pdl_wait();
+  // Only now may the second pass be scheduled: its CTAs read x before their own wait, which is
+  // safe because every CTA of this kernel has by then seen x complete.
+  pdl_launch_dependents();
   const int ni = Kg / 256;
   const uint64_t pol = l2_policy(true);                  // the second pass reads x again
   const int64_t first = first_segment<T>(x, segments, K, G, Kg, false, pol, &counter, stage);
@@ -321,10 +323,12 @@ rows_tensor_codes(const T* __restrict__ x, int64_t segments, int64_t K, int G, i
   if (threadIdx.x == 0) counter = 0;
   pdl_launch_dependents();
   __syncthreads();
-  pdl_wait();
   const int ni = Kg / 256;
   const uint64_t pol = l2_policy(false);
-  const int64_t first = first_segment<T>(x, segments, K, G, Kg, true, pol, &counter, stage);   // in flight during the fold
+  // x was complete before the first pass let this kernel be scheduled (see there), so the first
+  // copies start before the wait for the first pass's records and extremes.
+  const int64_t first = first_segment<T>(x, segments, K, G, Kg, true, pol, &counter, stage);
+  pdl_wait();
   for (int g = warp; g < G; g += kRowWarps) {
     unsigned long long lo = ~0ull, hi = 0ull;
     for (int c = lane; c < stat_ctas; c += 32) {
