@@ -75,7 +75,8 @@ typedef enum {
   BL_OP_FORWARD = 2,
   BL_OP_MATMUL_I32 = 3,
   BL_OP_MATMUL_DEQUANT = 4,
-  BL_OP_BLOCK_FORWARD = 5    /* M = batch * seq tokens, N = ffn width, K = model width d, G ignored (1) */
+  BL_OP_BLOCK_FORWARD = 5,   /* M = batch * seq tokens, N = ffn width, K = model width d, G ignored (1) */
+  BL_OP_FORWARD_LATENT = 6
 } bl_op;
 
 /* Human-readable name of a status code (static string, never NULL). */
@@ -157,6 +158,21 @@ bl_status bitlinear_forward(const void* x, bl_dtype xt, int64_t M, int64_t K, in
                             int eta_correction, const uint8_t* W_packed, bl_layout layout,
                             const float* beta, const int32_t* rowsum, void* y, bl_dtype yt,
                             void* ws, size_t ws_bytes, void* stream);
+
+/* The layer as it runs in training (Sec. 2.2, "mixed precision training": the latent weights are
+ * binarised on the fly during the forward pass): Eq. 1-3 on the high-precision W of this step,
+ * then Eq. 11, in one call.  Nothing of the packed form outlives the call except what the caller
+ * asks back.
+ *   W [N,K] of dtype wt (the latent weights).  Other arguments as for bitlinear_forward.
+ *   alpha_out, beta_out  NULL or fp32 [G]: the alpha_g and beta_g of this step (the straight-through
+ *                        backward pass needs beta).
+ * The packed weights live in the workspace, in PREFILL order when the shape allows the tensor-core
+ * kernel (K % 128 == 0 per group), else CANONICAL.  y is bit-identical to bitlinear_binarize_pack
+ * followed by bitlinear_forward.  Workspace: BL_OP_FORWARD_LATENT. */
+bl_status bitlinear_forward_latent(const void* x, bl_dtype xt, const void* W, bl_dtype wt, int64_t M, int64_t K,
+                                   int64_t N, int G, int b, bl_quant_mode mode, bl_gran gran, float ln_eps,
+                                   int eta_correction, float* alpha_out, float* beta_out, void* y, bl_dtype yt,
+                                   void* ws, size_t ws_bytes, void* stream);
 
 /* Step 4 alone, Eq. 7: acc[g,m,n] = sum over k in group g of W~[n,k] . x_q[m,k], exact int32.
  * The parity hook for "accumulators are bit-exact when fed given codes".

@@ -19,6 +19,7 @@ ABSMAX, ETA = 0, 1
 PER_TENSOR, PER_TOKEN = 0, 1
 CANONICAL, PREFILL, DECODE = 0, 1, 2
 OP_BINARIZE_PACK, OP_QUANT_ACT, OP_FORWARD, OP_MATMUL_I32, OP_MATMUL_DEQUANT, OP_BLOCK_FORWARD = 0, 1, 2, 3, 4, 5
+OP_FORWARD_LATENT = 6
 MAX_GROUPS = 64
 NOALLOC_MAX_SEGMENTS = 16384
 ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_TOO_LARGE = 1, 2, 3, 4, 5, 6, 7, 8
@@ -29,6 +30,7 @@ EXPORTS = [
     "bitlinear_forward", "bitlinear_matmul_i32", "bitlinear_matmul_dequant", "bitlinear_gemv_decode",
     "bitlinear_attention_causal", "bitlinear_block_forward", "bitlinear_ws_status",
     "bitlinear_matmul_dequant_ex", "bitlinear_binarize_pack_nsplit", "bitlinear_gemv_decode_batch",
+    "bitlinear_forward_latent",
 ]
 
 _DTYPES = {torch.float32: F32, torch.float16: F16, torch.bfloat16: BF16}
@@ -84,6 +86,9 @@ def lib():
         L.bitlinear_matmul_dequant_ex.restype = ci
         L.bitlinear_matmul_dequant_ex.argtypes = [vp, i64, i64, i64, ci, ci, vp, vp, ci, vp, ci, vp, vp, vp, vp, ci,
                                                   vp, sz, vp]
+        L.bitlinear_forward_latent.restype = ci
+        L.bitlinear_forward_latent.argtypes = [vp, ci, vp, ci, i64, i64, i64, ci, ci, ci, ci, C.c_float, ci, vp, vp, vp,
+                                               ci, vp, sz, vp]
         L.bitlinear_gemv_decode_batch.restype = ci
         L.bitlinear_gemv_decode_batch.argtypes = [vp, ci, i64, i64, i64, ci, ci, ci, C.c_float, ci, vp, vp, vp, vp,
                                                   ci, vp]
@@ -254,6 +259,24 @@ def matmul_dequant(x_q, gamma, W_packed, beta, N, G=1, gran=PER_TOKEN, layout=CA
                                           _ptr(rowsum), _ptr(y), _dt(y), _ptr(ws), ws.numel(), _stream())
     _check(code, "bitlinear_matmul_dequant")
     return y
+
+
+def forward_latent(x, W, G=1, mode=ABSMAX, gran=PER_TOKEN, ln_eps=1e-5, eta_correction=False, out_dtype=None,
+                   b=8, y=None, ws=None):
+    """bitlinear_forward_latent.  x [M,K], latent W [N,K]; returns dict(y [M,N], alpha, beta [G], ws)."""
+    M, K = x.shape
+    N = W.shape[0]
+    dev = x.device
+    if y is None:
+        y = torch.empty((M, N), dtype=out_dtype or x.dtype, device=dev)
+    alpha = torch.empty(G, dtype=torch.float32, device=dev)
+    beta = torch.empty(G, dtype=torch.float32, device=dev)
+    ws = _ws(workspace_bytes(OP_FORWARD_LATENT, M, N, K, G), dev, ws)
+    code = lib().bitlinear_forward_latent(_ptr(x), _dt(x), _ptr(W), _dt(W), M, K, N, G, b, mode, gran,
+                                          float(ln_eps), 1 if eta_correction else 0, _ptr(alpha), _ptr(beta),
+                                          _ptr(y), _dt(y), _ptr(ws), ws.numel(), _stream())
+    _check(code, "bitlinear_forward_latent")
+    return dict(y=y, alpha=alpha, beta=beta, ws=ws)
 
 
 class _Epilogue(C.Structure):

@@ -55,6 +55,24 @@ ForwardWs carve_forward(int64_t M, int64_t N, int64_t K, int G) {
   return w;
 }
 
+struct LatentWs {                      // carving of the BL_OP_FORWARD_LATENT workspace
+  size_t pack, packed, alpha, beta, rowsum, forward, total;
+  bl_layout layout;
+};
+LatentWs carve_latent(int64_t M, int64_t N, int64_t K, int G) {
+  LatentWs w;
+  w.layout = gemm_tc_supported(M, K, N, G) ? BL_LAYOUT_PREFILL : BL_LAYOUT_CANONICAL;
+  size_t off = 0;
+  w.pack = off;    off += round256(pack_ws_bytes(G));
+  w.packed = off;  off += round256(w.layout == BL_LAYOUT_PREFILL ? (size_t)prefill_bytes(N, K) : (size_t)(N * (K / 8)));
+  w.alpha = off;   off += round256((size_t)G * sizeof(float));
+  w.beta = off;    off += round256((size_t)G * sizeof(float));
+  w.rowsum = off;  off += round256((size_t)N * (size_t)G * sizeof(int32_t));
+  w.forward = off; off += carve_forward(M, N, K, G).total;
+  w.total = off;
+  return w;
+}
+
 bl_status check_layout_for_gemm(bl_layout layout, int64_t M, int64_t K, int64_t N, int G) {
   if (layout == BL_LAYOUT_CANONICAL) return BL_OK;
   if (layout == BL_LAYOUT_PREFILL) return gemm_tc_supported(M, K, N, G) ? BL_OK : BL_ERR_SHAPE;
@@ -89,6 +107,7 @@ size_t bitlinear_workspace_bytes(bl_op op, int64_t M, int64_t N, int64_t K, int 
     case BL_OP_MATMUL_I32:
     case BL_OP_MATMUL_DEQUANT: return (M > 0 && N > 0) ? gemm_ws_total(M, N, G) : 0;
     case BL_OP_BLOCK_FORWARD: return (M > 0 && N > 0) ? carve_block(M, K, N).total : 0;
+    case BL_OP_FORWARD_LATENT: return (M > 0 && N > 0) ? carve_latent(M, N, K, G).total : 0;
   }
   return 0;
 }
@@ -286,6 +305,34 @@ bl_status bitlinear_forward(const void* x, bl_dtype xt, int64_t M, int64_t K, in
   a.scratch = base + w.status + kStatusBytes;
   cudaError_t e = (layout == BL_LAYOUT_PREFILL) ? launch_gemm_tc(a, s) : launch_gemm_simple(a, s);
   return e == cudaSuccess ? BL_OK : BL_ERR_CUDA;
+}
+
+bl_status bitlinear_forward_latent(const void* x, bl_dtype xt, const void* W, bl_dtype wt, int64_t M, int64_t K,
+                                   int64_t N, int G, int b, bl_quant_mode mode, bl_gran gran, float ln_eps,
+                                   int eta_correction, float* alpha_out, float* beta_out, void* y, bl_dtype yt,
+                                   void* ws, size_t ws_bytes, void* stream) {
+  if (!x || !W || !y) return BL_ERR_NULL;
+  if (M <= 0 || N <= 0) return BL_ERR_SHAPE;
+  bl_status st = check_kg(K, G);
+  if (st != BL_OK) return st;
+  const LatentWs c = carve_latent(M, N, K, G);
+  if (!ws || ws_bytes < c.total) return BL_ERR_WORKSPACE;
+  if (!aligned16(ws)) return BL_ERR_ALIGN;
+  char* base = reinterpret_cast<char*>(ws);
+  uint8_t* packed = reinterpret_cast<uint8_t*>(base + c.packed);
+  float* alpha = reinterpret_cast<float*>(base + c.alpha);
+  float* beta = reinterpret_cast<float*>(base + c.beta);
+  int32_t* rowsum = reinterpret_cast<int32_t*>(base + c.rowsum);
+  st = bitlinear_binarize_pack(W, wt, N, K, G, c.layout, nullptr, packed, alpha, beta, rowsum, base + c.pack,
+                               round256(pack_ws_bytes(G)), stream);
+  if (st != BL_OK) return st;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (alpha_out && cudaMemcpyAsync(alpha_out, alpha, (size_t)G * sizeof(float), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+    return BL_ERR_CUDA;
+  if (beta_out && cudaMemcpyAsync(beta_out, beta, (size_t)G * sizeof(float), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+    return BL_ERR_CUDA;
+  return bitlinear_forward(x, xt, M, K, N, G, b, mode, gran, ln_eps, eta_correction, packed, c.layout, beta, rowsum, y,
+                           yt, base + c.forward, c.total - c.forward, stream);
 }
 
 bl_status bitlinear_gemv_decode(const void* x, bl_dtype xt, int64_t K, int64_t N, int G, int b,

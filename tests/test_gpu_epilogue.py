@@ -105,3 +105,31 @@ def test_epilogue_argument_checks():
     with pytest.raises(B.BitLinearError) as e:          # NB must divide N
         B.binarize_pack_nsplit(W, 7)
     assert e.value.code == B.ERR_SHAPE
+
+
+@pytest.mark.parametrize("M,K,N,G,wdtype,mode,gran", [
+    (200, 512, 384, 1, "f32", "absmax", "tensor"),     # tensor-core path
+    (64, 1024, 256, 2, "bf16", "eta", "token"),        # grouped, 16-bit latent weights
+    (33, 1000, 70, 5, "f32", "eta", "tensor"),         # shape only the CUDA-core kernel takes
+])
+def test_forward_latent_is_pack_then_forward(M, K, N, G, wdtype, mode, gran):
+    omode = O.ETA if mode == "eta" else O.ABSMAX
+    ogran = B.PER_TOKEN if gran == "token" else B.PER_TENSOR
+    x = synth.make_x(M, K, torch.bfloat16, seed=M + K, outliers=False, relu=(mode == "eta")).to(DEV)
+    W = synth.make_w(N, K, DT[wdtype], seed=N).to(DEV)
+    corr = mode == "eta"
+    got = B.forward_latent(x, W, G=G, mode=omode, gran=ogran, eta_correction=corr, out_dtype=torch.float32)
+    lay = B.PREFILL if (K // G) % 128 == 0 else B.CANONICAL
+    w = B.binarize_pack(W, G=G, layout=lay)
+    want = B.forward(x, w["W_packed"], w["beta"], N, G=G, mode=omode, gran=ogran, layout=lay, rowsum=w["rowsum"],
+                     eta_correction=corr, out_dtype=torch.float32)
+    assert torch.equal(got["y"], want)
+    assert torch.equal(got["alpha"], w["alpha"]) and torch.equal(got["beta"], w["beta"])
+    # and against the oracle on the same latent weights
+    w_ref = O.binarize(W.float().cpu().numpy(), G=G)
+    ref = O.forward(as_f32_np(x), w_ref["bits"], w_ref["beta"], G=G, mode=omode,
+                    gran=O.PER_TOKEN if gran == "token" else O.PER_TENSOR, ln_eps=1e-5, rowsum=w_ref["rowsum"],
+                    eta_correction=corr)
+    rms = np.sqrt((ref["y"] ** 2).mean())
+    err = np.abs(got["y"].cpu().numpy().astype(np.float64) - ref["y"])
+    assert np.median(err) <= 1e-3 * rms and np.quantile(err, 0.999) <= 2e-2 * rms
