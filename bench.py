@@ -40,7 +40,7 @@ INT8_TO_BF16 = 2.0                                   # nominal dense int8 : bf16
 # one that was profiled: set it to None when the kernel changes, until the capture is redone.
 NCU_TRAFFIC = {
     "gemm_tc2_kernel": 54.1e6,                       # 36.3 MB read + 17.8 MB written (y largely still in L2)
-    "rows_tensor_stats + rows_tensor_codes": None,     # kernels rewritten since the last capture
+    "rows_tensor_fused": None,                         # set from the ncu capture of the committed kernel
     "gemv_decode_kernel": 8.45e6,
     "reduce_partials + sign_pack": 135.3e6,          # 67.1 + 0.4 and 67.1 + 0.7 MB
 }
@@ -257,17 +257,17 @@ def run_b200(args):
                          "in total, larger than L2"},
         "clocks": None,
         "e2e": e2e,
-        "gpu_launches": 3 * K_steps,
-        "kernels_per_step": ["rows_tensor_stats", "rows_tensor_codes", "gemm_tc2_kernel"],
+        "gpu_launches": 2 * K_steps,
+        "kernels_per_step": ["rows_tensor_fused", "gemm_tc2_kernel"],
         "roofline": {"bound": "tensor", "kernel": "gemm_tc2_kernel", "achieved": gemm_tops, "peak": tensor_peak,
                      "unit": "TFLOP/s", "frac": gemm_tops / tensor_peak, "traffic": NCU_TRAFFIC["gemm_tc2_kernel"],
                      "op_kind": "int8 (s8 x s8 -> s32), 2 ops per multiply-accumulate",
                      "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} x {INT8_TO_BF16} "
                                     "(nominal int8:bf16 ratio)",
                      "frac_of_nominal": gemm_tops / NOMINAL_INT8_TOPS, "avg_launch_ms": gemm_ms},
-        "roofline_quant": {"bound": "hbm", "kernel": "rows_tensor_stats + rows_tensor_codes", "achieved": quant_gbs,
+        "roofline_quant": {"bound": "hbm", "kernel": "rows_tensor_fused", "achieved": quant_gbs,
                            "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": quant_gbs / peaks["hbm_gbs"],
-                           "traffic": NCU_TRAFFIC["rows_tensor_stats + rows_tensor_codes"], "avg_ms": quant_ms, "peak_source": peaks["source"] + " copy"},
+                           "traffic": NCU_TRAFFIC["rows_tensor_fused"], "avg_ms": quant_ms, "peak_source": peaks["source"] + " copy"},
     }
 
     parts = set(args.parts.split(","))

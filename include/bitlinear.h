@@ -114,7 +114,10 @@ bl_status bitlinear_binarize_pack(const void* W, bl_dtype wt, int64_t N, int64_t
  *   ln_eps LN epsilon; a negative value skips LN (codes are taken from x itself).
  *   x_q    int8 [M,K] codes.   gamma, eta: fp32, sized by gran (eta may be NULL for BL_ABSMAX).
  * gamma == 0 (constant input) yields all-zero codes, never NaN.  PER_TOKEN is one pass over x;
- * PER_TENSOR is two (statistics, then codes).  Workspace: BL_OP_QUANT_ACT. */
+ * PER_TENSOR is two (statistics, then codes).  For segments of up to 8 KB that are a multiple of
+ * 256 features both passes run in one cooperative kernel whose CTAs wait for one another between
+ * the passes, with a limit: after a PER_TENSOR call bitlinear_ws_status(ws, stream) reports
+ * BL_ERR_TIMEOUT if that wait expired (codes are then not written).  Workspace: BL_OP_QUANT_ACT. */
 bl_status bitlinear_quant_act(const void* x, bl_dtype xt, int64_t M, int64_t K, int G, int b,
                               bl_quant_mode mode, bl_gran gran, float ln_eps, int8_t* x_q,
                               float* gamma, float* eta, void* ws, size_t ws_bytes, void* stream);

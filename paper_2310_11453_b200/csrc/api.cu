@@ -296,8 +296,12 @@ bl_status bitlinear_forward(const void* x, bl_dtype xt, int64_t M, int64_t K, in
   float* gamma = reinterpret_cast<float*>(base + w.gamma);
   float* eta = reinterpret_cast<float*>(base + w.eta);
   QuantArgs q{x, xt, M, K, G, mode, gran, ln_eps, codes, gamma, eta, base + w.quant};
+  // One status word for the call: the per-tensor quant kernels clear it (and may report a timeout
+  // of their own), so the GEMM that follows must not clear it again.
+  q.status = reinterpret_cast<uint32_t*>(base + w.status);
   if (launch_quant_act(q, s) != cudaSuccess) return BL_ERR_CUDA;
   GemmArgs a{};
+  a.keep_status = gran == BL_PER_TENSOR ? 1 : 0;
   a.x_q = codes; a.M = M; a.K = K; a.N = N; a.G = G; a.W_packed = W_packed; a.acc = nullptr;
   a.y = y; a.yt = yt; a.beta = beta; a.gamma = gamma; a.eta = eta; a.gran = gran;
   a.rowsum = rowsum; a.eta_correction = eta_correction ? 1 : 0;

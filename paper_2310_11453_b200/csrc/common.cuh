@@ -145,6 +145,8 @@ cudaError_t launch_binarize_pack(const PackArgs& a, cudaStream_t s);
 struct QuantArgs {
   const void* x; bl_dtype xt; int64_t M, K; int G; bl_quant_mode mode; bl_gran gran; float ln_eps;
   int8_t* x_q; float* gamma; float* eta; void* ws;
+  uint32_t* status = nullptr;                      // word for a device-side timeout (per-tensor scope);
+                                                   // nullptr: the first word of ws
 };
 size_t quant_ws_bytes(int64_t M, int G);
 cudaError_t launch_quant_act(const QuantArgs& a, cudaStream_t s);
@@ -164,6 +166,7 @@ struct GemmArgs {
   const void* residual; int64_t ld_res;            // y += residual[m, n] (dtype yt, row stride ld_res)
   int64_t ld_y;                                    // row stride of y in elements (0: N)
   uint32_t* status;                                // device status word (tensor-core path)
+  int keep_status;                                 // the kernel before this one already cleared it
   void* scratch;                                   // gemm_tc_scratch_bytes(G) bytes (tensor-core path)
 };
 cudaError_t launch_gemm_simple(const GemmArgs& a, cudaStream_t s);

@@ -193,7 +193,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
   // Everything above touched only this cluster's shared and tensor memory, so it may overlap the
   // end of the kernel before this one on the stream; from here on global memory is read.
   pdl_wait();
-  if (blockIdx.x == 0 && threadIdx.x == 0) *a.status = 0u;   // a timeout (seconds later) overwrites it
+  if (blockIdx.x == 0 && threadIdx.x == 0 && !a.keep_status) *a.status = 0u;   // a timeout (seconds later) overwrites it
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer (own codes)

@@ -11,7 +11,9 @@
 // Per-tensor scope splits in two kernels: the first leaves each segment's moments in the
 // workspace and folds the extremes of x^ into a global atomic min/max on an order-preserving
 // encoding (order-independent, hence deterministic); the second re-reads x and writes codes.
+#include <atomic>
 #include <mutex>
+#include <random>
 #include <type_traits>
 
 #include "quant_rows.cuh"
@@ -37,9 +39,13 @@ struct ScopePartial {              // one CTA's extremes of x^ for one group (fa
   unsigned long long lo, hi;
 };
 constexpr int kMaxStatCtas = 256;  // upper bound on the grid of the persistent fast-path kernels
-// Per-tensor workspace: TensorScope | ScopePartial[kMaxStatCtas][BL_MAX_GROUPS] | SegRecord[M*G].
-constexpr size_t kWsHeaderBytes =
-    sizeof(TensorScope) + (size_t)kMaxStatCtas * BL_MAX_GROUPS * sizeof(ScopePartial);
+// Per-tensor workspace:
+//   status word (256 bytes reserved) | TensorScope | ScopePartial[kMaxStatCtas][BL_MAX_GROUPS] |
+//   arrival tags u64[kMaxStatCtas] | SegRecord[M*G].
+constexpr size_t kWsScopeOff = 256;
+constexpr size_t kWsPartialOff = kWsScopeOff + sizeof(TensorScope);
+constexpr size_t kWsTagOff = kWsPartialOff + (size_t)kMaxStatCtas * BL_MAX_GROUPS * sizeof(ScopePartial);
+constexpr size_t kWsHeaderBytes = kWsTagOff + (size_t)kMaxStatCtas * sizeof(unsigned long long);
 
 template <typename T>
 __device__ __forceinline__ void stage_segment(const T* __restrict__ src, int Kg, float* seg) {
@@ -82,8 +88,9 @@ quant_per_token(const T* __restrict__ x, int64_t K, int G, int mode, float ln_ep
   }
 }
 
-__global__ void init_scope(TensorScope* sc) {
+__global__ void init_scope(TensorScope* sc, uint32_t* status) {
   const int g = threadIdx.x;
+  if (g == 0) *status = 0u;                          // these kernels have no device-side wait
   if (g < BL_MAX_GROUPS) { sc->enc_min[g] = ~0ull; sc->enc_max[g] = 0ull; }
 }
 
@@ -280,7 +287,7 @@ rows_per_token(const T* __restrict__ x, int64_t segments, int64_t K, int G, int 
 template <typename T>
 __global__ void __launch_bounds__(kRowWarps * 32, 1)
 rows_tensor_stats(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg, float ln_eps, double inv_kg,
-                  ScopePartial* __restrict__ partials, SegRecord* __restrict__ recs) {
+                  ScopePartial* __restrict__ partials, SegRecord* __restrict__ recs, uint32_t* status) {
   extern __shared__ __align__(16) unsigned char stage[];
   __shared__ int counter;
   __shared__ unsigned long long part_lo[BL_MAX_GROUPS], part_hi[BL_MAX_GROUPS];
@@ -292,6 +299,7 @@ rows_tensor_stats(const T* __restrict__ x, int64_t segments, int64_t K, int G, i
   // Only now may the second pass be scheduled: its CTAs read x before their own wait, which is
   // safe because every CTA of this kernel has by then seen x complete.
   pdl_launch_dependents();
+  if (blockIdx.x == 0 && threadIdx.x == 0) *status = 0u;   // the two-kernel path has no device-side wait
   const int ni = Kg / 256;
   const uint64_t pol = l2_policy(true);                  // the second pass reads x again
   const int64_t first = first_segment<T>(x, segments, K, G, Kg, false, pol, &counter, stage);
@@ -359,6 +367,243 @@ rows_tensor_codes(const T* __restrict__ x, int64_t segments, int64_t K, int G, i
   });
 }
 
+// ---- per-tensor scope in one kernel ------------------------------------------------------------------
+// Both passes in one cooperative launch (every CTA is resident, so they can wait for one another).
+// Pass 1 as in rows_tensor_stats, except that the last two segments of every warp are handed out
+// statically: they are still in the warp's two slots when the pass ends.  Then the CTAs meet: each
+// publishes a tag (unique to the call, so the array needs no clearing) after its partial extremes,
+// and waits, with a limit, until all tags of the grid show it.  Pass 2 codes the retained segments
+// straight from shared memory (2 x 12 per SM that are not read from HBM again) and then the rest of
+// its range backwards, as rows_tensor_codes does.
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_u64(unsigned long long* p, unsigned long long v) {
+  asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+constexpr unsigned kMeetSpins = 1u << 22;                     // polls of the arrival tags before giving up
+constexpr unsigned long long kMeetNs = 2000000000ull;         // and a 2 s limit on the clock
+
+template <typename T>
+__global__ void __launch_bounds__(kRowWarps * 32, 1)
+rows_tensor_fused(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg, int mode, float ln_eps,
+                  double inv_kg, ScopePartial* __restrict__ partials, SegRecord* __restrict__ recs,
+                  unsigned long long* __restrict__ tags, unsigned long long tag, uint32_t* __restrict__ status,
+                  int8_t* __restrict__ x_q, float* __restrict__ gamma, float* __restrict__ eta) {
+  extern __shared__ __align__(16) unsigned char stage[];
+  __shared__ int counter1, counter2;
+  __shared__ unsigned long long part_lo[BL_MAX_GROUPS], part_hi[BL_MAX_GROUPS];
+  __shared__ double gam_s[BL_MAX_GROUPS], eta_s[BL_MAX_GROUPS];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint4* slots = reinterpret_cast<uint4*>(stage + (size_t)warp * 2 * kSlotBytes);
+  if (threadIdx.x == 0) { counter1 = 0; counter2 = 0; }
+  if (threadIdx.x < BL_MAX_GROUPS) { part_lo[threadIdx.x] = ~0ull; part_hi[threadIdx.x] = 0ull; }
+  __syncthreads();
+  pdl_wait();
+  pdl_launch_dependents();
+  if (blockIdx.x == 0 && threadIdx.x == 0) *status = 0u;        // a timeout (seconds later) overwrites it
+
+  const RowRange rg = cta_range(segments);
+  const int n = (int)(rg.end - rg.begin);
+  const int n_keep = n < 2 * kRowWarps ? n : 2 * kRowWarps;     // handed out statically, stay in the slots
+  const int n_dyn = n - n_keep;                                 // drawn through the counters
+  const int ni = Kg / 256;
+  const int nv = ni * RowTraits<T>::kVecPerChunk;               // 16-byte pieces per lane
+  auto issue = [&](int64_t seg, uint4* slot, uint64_t policy) {
+    if (seg >= 0) {
+      const uint4* src = reinterpret_cast<const uint4*>(x + (seg / G) * K + (seg % G) * (int64_t)Kg);
+#pragma unroll 4
+      for (int i = 0; i < nv; ++i) cp_async16(slot + lane + 32 * i, src + lane + 32 * i, policy);
+    }
+    cp_async_commit();
+  };
+  auto slot_of = [&](int c) { return slots + c * (kSlotBytes / 16); };
+
+  // ---- pass 1
+  bool dyn_done = n_dyn == 0;
+  int statics = 0;
+  auto draw1 = [&]() -> int64_t {
+    if (!dyn_done) {
+      int r = 0;
+      if (lane == 0) r = atomicAdd(&counter1, 1);
+      r = __shfl_sync(0xFFFFFFFFu, r, 0);
+      if (r < n_dyn) return rg.begin + r;
+      dyn_done = true;
+    }
+    const int j = warp + kRowWarps * statics;
+    if (j < n_keep) { ++statics; return rg.begin + n_dyn + j; }
+    return -1;
+  };
+  const uint64_t keep = l2_policy(true), last_use = l2_policy(false);
+  int cur = 0;
+  int64_t seg = draw1();
+  issue(seg, slot_of(0), keep);
+  int64_t seg_last = -1, seg_prev = -1;
+  RowStats st_last = {0.0, 0.0, 0.f, 0.f}, st_prev = st_last;
+  while (seg >= 0) {
+    const int64_t next = draw1();
+    issue(next, slot_of(cur ^ 1), next >= rg.begin + n_dyn ? last_use : keep);
+    cp_async_wait_but_newest();
+    __syncwarp();
+    const RowStats st = row_stats<T>(slot_of(cur), ni, lane, ln_eps, inv_kg);
+    if (lane == 0) {
+      const int g = (int)(seg % G);
+      recs[seg] = SegRecord{st.mean, st.rstd, st.xlo, st.xhi};
+      atomicMin(&part_lo[g], enc_ordered64(((double)st.xlo - st.mean) * st.rstd));
+      atomicMax(&part_hi[g], enc_ordered64(((double)st.xhi - st.mean) * st.rstd));
+    }
+    __syncwarp();
+    seg_prev = seg_last; st_prev = st_last;
+    seg_last = seg; st_last = st;
+    seg = next;
+    if (seg >= 0) cur ^= 1;                                     // cur stays on the last segment's slot
+  }
+  // retained: seg_last in slot cur, and (if the warp had two static draws) seg_prev in slot cur ^ 1
+  const int kept = statics;                                      // 0, 1 or 2
+  __syncthreads();
+  if (threadIdx.x < G)
+    partials[(size_t)blockIdx.x * G + threadIdx.x] = ScopePartial{part_lo[threadIdx.x], part_hi[threadIdx.x]};
+  __syncthreads();
+
+  // ---- the CTAs meet
+  if (threadIdx.x == 0) { __threadfence(); st_release_u64(tags + blockIdx.x, tag); }
+  bool here = true;
+  if (threadIdx.x < gridDim.x) {
+    here = false;
+    unsigned long long t0 = 0;
+    for (unsigned it = 0; it < kMeetSpins; ++it) {
+      if (ld_acquire_u64(tags + threadIdx.x) == tag) { here = true; break; }
+      if ((it & 63u) == 63u) {
+        unsigned long long now;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+        if (t0 == 0) t0 = now;
+        else if (now - t0 > kMeetNs) break;
+      }
+      __nanosleep(64);
+    }
+  }
+  if (!__syncthreads_and(here)) {                                // someone never arrived: codes are not written
+    if (threadIdx.x == 0) atomicExch(status, (uint32_t)BL_ERR_TIMEOUT);
+    return;
+  }
+
+  // ---- gamma / eta of every group from all CTAs' extremes
+  for (int g = warp; g < G; g += kRowWarps) {
+    unsigned long long lo = ~0ull, hi = 0ull;
+    for (int c = lane; c < (int)gridDim.x; c += 32) {
+      const ScopePartial p = partials[(size_t)c * G + g];
+      lo = min(lo, p.lo); hi = max(hi, p.hi);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      lo = min(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, o));
+      hi = max(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, o));
+    }
+    if (lane == 0) {
+      double gam, et;
+      scope_gamma_eta(mode, dec_ordered64(lo), dec_ordered64(hi), gam, et);
+      gam_s[g] = gam; eta_s[g] = et;
+      if (blockIdx.x == 0) {
+        gamma[g] = (float)gam;
+        if (eta) eta[g] = (float)et;
+      }
+    }
+  }
+  __syncthreads();
+
+  // ---- pass 2
+  auto code = [&](int64_t sg, const RowStats& st, const uint4* slot) {
+    const int g = (int)(sg % G);
+    const RowMap map = row_map(mode, st.mean, st.rstd, gam_s[g], eta_s[g], st.xlo, st.xhi);
+    row_store_codes<T>(slot, ni, lane, map, x_q + (sg / G) * K + g * (int64_t)Kg);
+  };
+  auto draw2 = [&]() -> int64_t {
+    int r = 0;
+    if (lane == 0) r = atomicAdd(&counter2, 1);
+    r = __shfl_sync(0xFFFFFFFFu, r, 0);
+    return r < n_dyn ? rg.begin + n_dyn - 1 - r : -1;           // backwards: the rows read last first
+  };
+  if (kept >= 1) code(seg_last, st_last, slot_of(cur));
+  __syncwarp();
+  seg = n_dyn > 0 ? draw2() : -1;
+  issue(seg, slot_of(cur), last_use);                            // overlaps the second retained segment
+  if (kept >= 2) code(seg_prev, st_prev, slot_of(cur ^ 1));
+  __syncwarp();
+  while (seg >= 0) {
+    const int64_t next = draw2();
+    issue(next, slot_of(cur ^ 1), last_use);
+    const SegRecord rec = recs[seg];
+    cp_async_wait_but_newest();
+    __syncwarp();
+    code(seg, RowStats{rec.mean, rec.rstd, rec.xlo, rec.xhi}, slot_of(cur));
+    __syncwarp();
+    seg = next; cur ^= 1;
+  }
+  asm volatile("cp.async.wait_all;" ::: "memory");
+}
+
+// Unique, never zero, per call: high half drawn once per process, low half a call counter.
+inline unsigned long long next_tag() {
+  static const unsigned long long high = [] {
+    std::random_device rd;
+    return ((unsigned long long)rd() << 32) ^ ((unsigned long long)rd() << 13);
+  }();
+  static std::atomic<unsigned long long> calls{1};
+  const unsigned long long t = (high & 0xFFFFFFFF00000000ull) | (calls.fetch_add(1) & 0xFFFFFFFFull);
+  return t ? t : 1;
+}
+
+// cudaErrorNotSupported: the device or context cannot launch cooperatively (the caller falls back).
+template <typename T>
+cudaError_t launch_fused(const QuantArgs& a, cudaStream_t s, const T* x, int64_t segments, int Kg, double inv_kg,
+                         unsigned grid, ScopePartial* partials, SegRecord* recs, uint32_t* status) {
+  int dev = 0, coop = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) return cudaErrorNotSupported;
+  auto kern = rows_tensor_fused<T>;
+  if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowStage)) != cudaSuccess) return e;
+  // CTAs that can be resident at once on this device (cached per device ordinal)
+  static std::atomic<int> resident[64] = {};
+  int cap = dev < 64 ? resident[dev].load() : 0;
+  if (cap == 0) {
+    int per_sm = 0, sms = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kRowWarps * 32, kRowStage) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || per_sm < 1)
+      return cudaErrorNotSupported;
+    cap = per_sm * sms;
+    if (dev < 64) resident[dev].store(cap);
+  }
+  if ((int64_t)grid > (int64_t)cap) grid = (unsigned)cap;
+  unsigned long long* tags = reinterpret_cast<unsigned long long*>(reinterpret_cast<char*>(a.ws) + kWsTagOff);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kRowWarps * 32);
+  cfg.dynamicSmemBytes = kRowStage;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeCooperative;
+  attr[0].val.cooperative = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  static std::atomic<int> with_pdl{1};                          // dropped for good if the pair is refused once
+  cfg.numAttrs = with_pdl.load() ? 2 : 1;
+  const unsigned long long tag = next_tag();
+  e = cudaLaunchKernelEx(&cfg, kern, x, segments, a.K, a.G, Kg, (int)a.mode, a.ln_eps, inv_kg, partials, recs, tags,
+                         tag, status, a.x_q, a.gamma, a.eta);
+  if (e != cudaSuccess && cfg.numAttrs == 2) {
+    (void)cudaGetLastError();
+    with_pdl.store(0);
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, kern, x, segments, a.K, a.G, Kg, (int)a.mode, a.ln_eps, inv_kg, partials, recs, tags,
+                           tag, status, a.x_q, a.gamma, a.eta);
+  }
+  return e;
+}
+
 // Grid of the persistent kernels: one CTA per SM, never more CTAs than segments.
 inline cudaError_t rows_grid(int64_t segments, unsigned* grid) {
   int dev = 0, sms = 0;
@@ -388,12 +633,18 @@ cudaError_t run_rows(const QuantArgs& a, cudaStream_t s) {
     return launch_pdl(rows_per_token<T>, grid, kThreads, kRowStage, s, x, segments, a.K, a.G, Kg, (int)a.mode,
                       a.ln_eps, inv_kg, a.x_q, a.gamma, a.eta);
   }
-  ScopePartial* partials = reinterpret_cast<ScopePartial*>(reinterpret_cast<char*>(a.ws) + sizeof(TensorScope));
+  ScopePartial* partials = reinterpret_cast<ScopePartial*>(reinterpret_cast<char*>(a.ws) + kWsPartialOff);
   SegRecord* recs = reinterpret_cast<SegRecord*>(reinterpret_cast<char*>(a.ws) + kWsHeaderBytes);
+  uint32_t* status = a.status ? a.status : reinterpret_cast<uint32_t*>(a.ws);
+  if (Kg * (int)sizeof(T) <= kSlotBytes) {                       // two slots per warp: both passes in one kernel
+    e = launch_fused<T>(a, s, x, segments, Kg, inv_kg, grid, partials, recs, status);
+    if (e != cudaErrorNotSupported) return e;                    // no cooperative launch here: two kernels
+    (void)cudaGetLastError();
+  }
   if ((e = cudaFuncSetAttribute(rows_tensor_stats<T>, attr, kRowStage)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(rows_tensor_codes<T>, attr, kRowStage)) != cudaSuccess) return e;
   e = launch_pdl(rows_tensor_stats<T>, grid, kThreads, kRowStage, s, x, segments, a.K, a.G, Kg, a.ln_eps, inv_kg,
-                 partials, recs);
+                 partials, recs, status);
   if (e != cudaSuccess) return e;
   return launch_pdl(rows_tensor_codes<T>, grid, kThreads, kRowStage, s, x, segments, a.K, a.G, Kg, (int)a.mode,
                     (int)grid, (const ScopePartial*)partials, (const SegRecord*)recs, a.x_q, a.gamma, a.eta);
@@ -417,13 +668,13 @@ cudaError_t run(const QuantArgs& a, cudaStream_t s) {
                                                         a.gamma, a.eta);
     return cudaGetLastError();
   }
-  TensorScope* sc = reinterpret_cast<TensorScope*>(a.ws);
+  TensorScope* sc = reinterpret_cast<TensorScope*>(reinterpret_cast<char*>(a.ws) + kWsScopeOff);
   SegRecord* recs = reinterpret_cast<SegRecord*>(reinterpret_cast<char*>(a.ws) + kWsHeaderBytes);
   if (smem > 48 * 1024) {
     e = cudaFuncSetAttribute(tensor_stats<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  init_scope<<<1, BL_MAX_GROUPS, 0, s>>>(sc);
+  init_scope<<<1, BL_MAX_GROUPS, 0, s>>>(sc, a.status ? a.status : reinterpret_cast<uint32_t*>(a.ws));
   tensor_stats<T><<<grid, kQuantThreads, smem, s>>>(x, a.K, a.G, a.ln_eps, sc, recs);
   tensor_codes<T><<<grid, kQuantThreads, 0, s>>>(x, a.K, a.G, (int)a.mode, sc, recs, a.x_q, a.gamma, a.eta);
   return cudaGetLastError();
