@@ -6,6 +6,7 @@ import torch
 from oracle import oracle as O
 from paper_2310_11453_b200 import binding as B
 from paper_2310_11453_b200 import synth
+from tests.test_gpu_parity import count_exact_ties
 from tests.util import as_f32_np
 
 pytestmark = pytest.mark.gpu
@@ -28,7 +29,11 @@ def test_gemv_decode_batch(M, K, N, G, dtype, mode, relu):
     w_ref = O.binarize(W.numpy(), G=G)
     w_gpu = B.binarize_pack(W.to(DEV), G=G, layout=B.DECODE)
     xd = x.to(DEV)
-    # the kernel's LN + Quant is the per-token path of bitlinear_quant_act: same codes, gamma, eta
+    # The kernel quantises the tokens itself and its codes cannot be read back, so the comparison
+    # allows what the quantising kernels are allowed: a different neighbour at a rounding tie,
+    # exact rational ties of the per-token eta form (either neighbour is valid) and, as for every
+    # quantising kernel here, at most 1e-4 of the elements (at least one).  Each such code moves a
+    # token's outputs by one quantisation step.
     q = B.quant_act(xd, G=G, mode=omode, gran=B.PER_TOKEN, ln_eps=1e-5)
     ref_q = O.quant_act(as_f32_np(x), G=G, mode=omode, gran=O.PER_TOKEN, ln_eps=1e-5)
     codes = q["x_q"].cpu().numpy()
@@ -43,7 +48,13 @@ def test_gemv_decode_batch(M, K, N, G, dtype, mode, relu):
                          q["gamma"].cpu().numpy().astype(np.float64), gran=O.PER_TOKEN,
                          eta=q["eta"].cpu().numpy().astype(np.float64), rowsum=w_ref["rowsum"], eta_correction=corr)
         rms = np.sqrt((want ** 2).mean())
-        assert np.abs(y.cpu().numpy().astype(np.float64) - want).max() <= 1e-3 * rms
+        gam = q["gamma"].cpu().numpy().astype(np.float64).reshape(M, G)
+        step = (w_gpu["beta"].cpu().numpy().astype(np.float64)[None, :] * gam / 128.0).max(axis=1)
+        ties = np.array([count_exact_ties(as_f32_np(x)[m], G) if mode == "eta" else 0 for m in range(M)])
+        slack = ((max(1, int(1e-4 * K)) + ties) * step)[:, None]
+        err = np.abs(y.cpu().numpy().astype(np.float64) - want)
+        assert (err <= 1e-3 * rms + slack).all()
+        assert np.median(err) <= 1e-3 * rms                      # the typical element needs no slack
     # 16-bit output is the rounding of the fp32 one
     y32 = B.gemv_decode_batch(xd, w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode, out_dtype=torch.float32)
     if dtype != "f32":
