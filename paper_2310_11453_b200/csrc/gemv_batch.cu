@@ -2,25 +2,27 @@
 // per-token gamma), LN + Quant of the tokens (Eq. 12, 4-6) fused in front.  Bound by streaming the
 // packed weights (N*K/8 bytes) once; the tokens and outputs are a few hundred KB.
 //
-// Shape of one call.  A CTA has 8 warps.
-//   1. Every warp loads the packed weights of its first two batches of K blocks into registers
-//      (they do not depend on x), lets the next kernel on the stream be scheduled and waits for
-//      everything earlier on the stream (programmatic dependent launch).
-//   2. Warp t normalises and quantises token t (every CTA does all tokens: 8 x K values out of
-//      L2, cheaper than a separate launch) and leaves the int8 codes in shared memory, one padded
-//      row per token, with the per-group sums of the codes, gamma and eta.  A group segment of up
-//      to 8 KB is first copied to the warp's staging slot with all its asynchronous copies in
-//      flight at once, so the two passes over it (statistics, codes) run at shared-memory
-//      latency; longer segments are read from L2 twice.
-//   3. Per 16 rows, the warp runs the 1-bit x 8-bit product on the tensor cores without ever
-//      expanding the weights to bytes.  DECODE layout puts weight q of a 32-weight word at bit
-//      q/4 + 8*(q%4), so word & (0x01010101 << j) is four bytes that are 0 or 2^j, the
-//      weights 4j..4j+3 of the word.  Eight such words of a row (256 weights) are one 16 x 32
-//      byte A operand per bit plane j (one logic instruction per register), the tokens' matching
-//      codes the 32 x 8 B operand, and mma.sync m16n8k32 (s8 x s8 -> s32) accumulates
-//      2^j * sum_{bit = 1} x~ for 16 rows x 8 tokens (-2^7 for plane 7, whose byte 0x80 reads as
-//      -128).  Planes keep separate accumulators (eight independent chains); a group's result is
-//      sum_j |acc_j| >> j, exact, and sum_k W~ x~ = 2 * (that) - sum_k x~.
+// Shape of one call.  One CTA of 16 warps per SM.
+//   1. Every warp loads its first two batches of packed-weight blocks into registers (they do not
+//      depend on x), lets the next kernel on the stream be scheduled and waits for everything
+//      earlier on the stream (programmatic dependent launch).
+//   2. The tokens are copied to shared memory (all asynchronous copies in flight at once) and
+//      quantised there, 16 / M' warps per token (M' = M rounded up to a power of two): each warp
+//      takes every P-th row of 256 elements of a group segment, the warps of a token meet at a
+//      named barrier to add up their partial sums, and each writes the codes of its rows to the
+//      token's padded row of int8 codes in shared memory.  Every CTA does all tokens (8 x K values
+//      out of L2: cheaper than a separate launch).
+//   3. Two warps share a tile of 16 output rows, each taking half of the K blocks of every group.
+//      The 1-bit x 8-bit product runs on the tensor cores without ever expanding the weights to
+//      bytes.  DECODE layout puts weight q of a 32-weight word at bit q/4 + 8*(q%4), so
+//      word & (0x01010101 << j) is four bytes that are 0 or 2^j, the weights 4j..4j+3 of the word.
+//      Eight such words of a row (256 weights) are one 16 x 32 byte A operand per bit plane j (one
+//      logic instruction per register), the tokens' matching codes the 32 x 8 B operand, and
+//      mma.sync m16n8k32 (s8 x s8 -> s32) accumulates 2^j * sum_{bit = 1} x~ for 16 rows x 8 tokens
+//      (-2^7 for plane 7, whose byte 0x80 reads as -128).  Planes keep separate accumulators (eight
+//      independent chains); sum_j |acc_j| >> j is exact.  At the end of a group the second warp of
+//      the pair hands its sums over through shared memory and the first one finishes:
+//      sum_k W~ x~ = 2 * (sum over set bits) - sum_k x~, then the rescale of Eq. 11.
 #include "quant_rows.cuh"
 
 namespace bl {
@@ -30,25 +32,33 @@ namespace {
 using namespace rows;
 
 constexpr int kBatchTokens = 8;          // tokens per launch = columns of the MMA
-constexpr int kBatchWarps = 8;
-constexpr int kTileRows = 16;            // output rows per warp tile = rows of the MMA
+constexpr int kBatchWarps = 16;
+constexpr int kPairs = kBatchWarps / 2;  // two warps per 16-row tile
+constexpr int kTileRows = 16;            // output rows per tile = rows of the MMA
 constexpr int kBlockK = 256;             // weights per row and MMA step: 8 words of 32
-constexpr int kPreload = 8;              // K blocks per batch; two batches are held in registers (2 x 8 x 4 words)
+constexpr int kPreload = 4;              // K blocks per batch; two batches are held in registers (2 x 4 x 4 words)
 constexpr int kRowPad = 16;              // bytes between token rows beyond K (bank spread of the B loads)
 constexpr int kZeroBytes = 64;           // zero area read by the lanes of absent tokens
-constexpr int kStageBytes = 8192;        // per-warp staging slot for one group segment of a token
+constexpr size_t kSmemBudget = 220 * 1024;
 
 struct BatchShared {
   int csum[kBatchTokens][BL_MAX_GROUPS];
   float gamma[kBatchTokens][BL_MAX_GROUPS];
   float eta[kBatchTokens][BL_MAX_GROUPS];
+  double part_s[kBatchWarps], part_q[kBatchWarps];   // per-warp partial sums of one group segment
+  float part_lo[kBatchWarps], part_hi[kBatchWarps];
+  int part_c[kBatchWarps];
+  int handover[kPairs][32][4];                       // second warp of a pair -> first, per group
 };
 
+// Named barrier `id` (1..15) for `threads` threads (a multiple of 32): a hardware barrier, no polling.
+__device__ __forceinline__ void bar_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
                "l"(gsrc) : "memory");
 }
-
 __device__ __forceinline__ void mma_s8s8(int (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm volatile(
       "mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
@@ -60,6 +70,8 @@ __device__ __forceinline__ void mma_s8s8(int (&d)[4], const uint32_t (&a)[4], ui
 struct BatchArgs {
   const void* x; int M; int64_t K, N; int G; int mode; float ln_eps; int eta_correction;
   const uint8_t* W_packed; const float* beta; const int32_t* rowsum; void* y;
+  int stage_tokens;                      // the raw tokens fit in shared memory beside the codes
+  double inv_kg;                         // 1 / K_g (a double-precision division per thread otherwise)
 };
 
 // The four A words of K block b for this lane: rows g and g + 8, words qd and 4 + qd of the block.
@@ -79,168 +91,234 @@ gemv_batch_kernel(BatchArgs a) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g8 = lane >> 2, qd = lane & 3;                   // MMA fragment coordinates
   const int Kg = (int)(a.K / a.G);
-  const int blocks_per_group = Kg / kBlockK;
+  const int bpg = Kg / kBlockK;                              // K blocks per group
   const int64_t stride = a.K + kRowPad;                      // bytes between token rows of codes
-  uint4* slot = reinterpret_cast<uint4*>(smem + kZeroBytes + (size_t)warp * kStageBytes);
-  int8_t* codes = reinterpret_cast<int8_t*>(smem + kZeroBytes + (size_t)kBatchWarps * kStageBytes);
+  int8_t* codes = reinterpret_cast<int8_t*>(smem + kZeroBytes);
+  unsigned char* raw = smem + kZeroBytes + (size_t)a.M * stride;   // staged tokens, [M][K] of TX
   const int64_t words_per_row = a.K / 32;
   const uint32_t* W32 = reinterpret_cast<const uint32_t*>(a.W_packed);
   const int64_t tiles = a.N / kTileRows;
 
-  // 1. the warp's first two batches of weight blocks into registers; these loads read only the
-  //    static weights.  Work items are (tile, batch): a batch is up to kPreload K blocks of one group.
-  const int nbg = (blocks_per_group + kPreload - 1) / kPreload;   // batches per group
-  const int nbt = a.G * nbg;                                      // batches per tile
-  const int64_t tile_step = (int64_t)gridDim.x * kBatchWarps;
-  struct Item { int64_t tile; int t; };
-  auto valid = [&](const Item& it) { return it.tile < tiles; };
+  // ---- 1. work of this warp in the rows phase: half h of every group's blocks of the pair's tiles
+  const int pair = warp >> 1, h = warp & 1;
+  const int half0 = (bpg + 1) / 2;
+  const int my_blocks = h == 0 ? half0 : bpg - half0;        // per group (may be 0 for h = 1)
+  const int my_first = h == 0 ? 0 : half0;
+  const int nbg = (my_blocks + kPreload - 1) / kPreload;     // my batches per group
+  const int64_t tile_step = (int64_t)gridDim.x * kPairs;
+  const int64_t tile0 = (int64_t)blockIdx.x + (int64_t)gridDim.x * pair;
+  struct Item { int64_t tile; int g, b; };
+  auto valid = [&](const Item& it) { return nbg > 0 && it.tile < tiles; };
   auto next = [&](const Item& it) {
     Item n = it;
-    if (++n.t == nbt) { n.t = 0; n.tile += tile_step; }
+    if (++n.b >= nbg) { n.b = 0; if (++n.g == a.G) { n.g = 0; n.tile += tile_step; } }
     return n;
-  };
-  // first K block and number of K blocks of a batch
-  auto first_block = [&](const Item& it) { return (it.t / nbg) * blocks_per_group + (it.t % nbg) * kPreload; };
-  auto num_blocks = [&](const Item& it) {
-    const int left = blocks_per_group - (it.t % nbg) * kPreload;
-    return left < kPreload ? left : kPreload;
   };
   auto load_item = [&](const Item& it, uint32_t (&w)[kPreload][4]) {
     const uint32_t* lo = W32 + (it.tile * kTileRows + g8) * words_per_row;
     const uint32_t* hi = lo + 8 * words_per_row;
-    const int b0 = first_block(it), nb = num_blocks(it);
+    const int b0 = it.g * bpg + my_first + it.b * kPreload;
+    const int left = my_blocks - it.b * kPreload;
+    const int nb = left < kPreload ? left : kPreload;
 #pragma unroll
     for (int i = 0; i < kPreload; ++i)
       if (i < nb) load_block(lo, hi, b0 + i, qd, w[i]);
   };
-  Item cur{(int64_t)blockIdx.x + (int64_t)gridDim.x * warp, 0};
-  Item nxt = next(cur);
+  Item it1{tile0, 0, 0};
+  Item it2 = next(it1);
   uint32_t wa[kPreload][4], wb[kPreload][4];
-  if (valid(cur)) load_item(cur, wa);
-  if (valid(nxt)) load_item(nxt, wb);
+  if (valid(it1)) load_item(it1, wa);
+  if (valid(it2)) load_item(it2, wb);
   if (threadIdx.x < kZeroBytes / 4) reinterpret_cast<uint32_t*>(smem)[threadIdx.x] = 0u;
   pdl_launch_dependents();
   pdl_wait();
 
-  // 2. LN + Quant of token `warp`
-  if (warp < a.M) {
-    const TX* xt = reinterpret_cast<const TX*>(a.x) + (int64_t)warp * a.K;
-    const int ni = Kg / 256;
-    const double inv_kg = 1.0 / (double)Kg;
-    const int pieces = Kg * (int)sizeof(TX) / 512;             // 16-byte pieces per lane
-    const bool staged = Kg * (int)sizeof(TX) <= kStageBytes;
-    for (int g = 0; g < a.G; ++g) {
-      const uint4* seg = reinterpret_cast<const uint4*>(xt + (int64_t)g * Kg);
-      if (staged) {
-        __syncwarp();                                           // the previous group's reads are done
-        for (int i = 0; i < pieces; ++i) cp_async16(slot + lane + 32 * i, seg + lane + 32 * i);
-        asm volatile("cp.async.wait_all;" ::: "memory");
-        __syncwarp();
-        seg = slot;
+  // ---- 2. LN + Quant of the tokens
+  if (a.stage_tokens) {
+    const uint4* src = reinterpret_cast<const uint4*>(a.x);
+    uint4* dst = reinterpret_cast<uint4*>(raw);
+    const int pieces = (int)((size_t)a.M * a.K * sizeof(TX) / 16);
+    for (int i = threadIdx.x; i < pieces; i += kBatchWarps * 32) cp_async16(dst + i, src + i);
+    asm volatile("cp.async.wait_all;" ::: "memory");
+  }
+  __syncthreads();
+  {
+    int mp = 1;
+    while (mp < a.M) mp <<= 1;
+    const int P = kBatchWarps / mp;                           // warps per token
+    const int tok = warp / P, j = warp % P, w0 = tok * P;
+    if (tok < a.M) {
+      const TX* xt = a.stage_tokens ? reinterpret_cast<const TX*>(raw) + (int64_t)tok * a.K
+                                    : reinterpret_cast<const TX*>(a.x) + (int64_t)tok * a.K;
+      const int rows_per_group = Kg / 256;                    // 32-chunk rows of a group segment
+      const double inv_kg = a.inv_kg;
+      for (int g = 0; g < a.G; ++g) {
+        const uint4* seg = reinterpret_cast<const uint4*>(xt + (int64_t)g * Kg);
+        float pilot;
+        {
+          Chunk<TX> ch; float v[8];
+          ch.load(seg, 0); ch.unpack(v);                      // same address in every thread: a broadcast
+          pilot = 0.125f * (((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7])));
+          if (a.ln_eps < 0.f) pilot = 0.f;
+        }
+        float sum = 0.f, sq = 0.f, mn = INFINITY, mx = -INFINITY;
+        for (int rr = j; rr < rows_per_group; rr += P) {
+          Chunk<TX> ch; float v[8], d[8];
+          ch.load(seg, rr * 32 + lane); ch.unpack(v);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) { d[i] = v[i] - pilot; mn = fminf(mn, v[i]); mx = fmaxf(mx, v[i]); }
+          sum += ((d[0] + d[1]) + (d[2] + d[3])) + ((d[4] + d[5]) + (d[6] + d[7]));
+          float p0 = d[0] * d[0], p1 = d[1] * d[1];
+#pragma unroll
+          for (int i = 2; i < 8; i += 2) { p0 = fmaf(d[i], d[i], p0); p1 = fmaf(d[i + 1], d[i + 1], p1); }
+          sq += p0 + p1;
+        }
+        const double S = warp_sum((double)sum), Q = warp_sum((double)sq);
+        mn = warp_min(mn); mx = warp_max(mx);
+        if (lane == 0) { sh.part_s[warp] = S; sh.part_q[warp] = Q; sh.part_lo[warp] = mn; sh.part_hi[warp] = mx; }
+        bar_sync(1 + tok, P * 32);
+        double St = 0.0, Qt = 0.0;
+        float xlo = INFINITY, xhi = -INFINITY;
+        for (int w = w0; w < w0 + P; ++w) {
+          St += sh.part_s[w]; Qt += sh.part_q[w];
+          xlo = fminf(xlo, sh.part_lo[w]); xhi = fmaxf(xhi, sh.part_hi[w]);
+        }
+        double mean = 0.0, rstd = 1.0;
+        if (!(a.ln_eps < 0.f)) {
+          const double dm = St * inv_kg;                      // mean - pilot
+          mean = (double)pilot + dm;
+          double var = Qt * inv_kg - dm * dm;
+          if (var < 0.0) var = 0.0;
+          rstd = rsqrt_newton(var + (double)a.ln_eps);
+        }
+        double gam, et;
+        scope_gamma_eta(a.mode, ((double)xlo - mean) * rstd, ((double)xhi - mean) * rstd, gam, et);
+        const RowMap map = row_map(a.mode, mean, rstd, gam, et, xlo, xhi);
+        int8_t* row = codes + (int64_t)tok * stride + (int64_t)g * Kg;
+        int cs = 0;
+        for (int rr = j; rr < rows_per_group; rr += P) {
+          const int c = rr * 32 + lane;
+          Chunk<TX> ch; float v[8];
+          ch.load(seg, c); ch.unpack(v);
+          const uint2 cd = map.clip ? row_codes8<true>(v, map) : row_codes8<false>(v, map);
+          cs = __dp4a((int)cd.x, 0x01010101, cs);
+          cs = __dp4a((int)cd.y, 0x01010101, cs);
+          *reinterpret_cast<uint2*>(row + (size_t)c * 8) = cd;
+        }
+        cs = warp_sum(cs);
+        if (lane == 0) sh.part_c[warp] = cs;
+        bar_sync(1 + tok, P * 32);
+        if (j == 0 && lane == 0) {
+          int tot = 0;
+          for (int w = w0; w < w0 + P; ++w) tot += sh.part_c[w];
+          sh.csum[tok][g] = tot; sh.gamma[tok][g] = (float)gam; sh.eta[tok][g] = (float)et;
+        }
+        bar_sync(1 + tok, P * 32);                            // the partial sums may be overwritten
       }
-      const RowStats st = row_stats<TX>(seg, ni, lane, a.ln_eps, inv_kg);
-      const double lo = ((double)st.xlo - st.mean) * st.rstd, hi = ((double)st.xhi - st.mean) * st.rstd;
-      double gam, et;
-      scope_gamma_eta(a.mode, lo, hi, gam, et);
-      const RowMap map = row_map(a.mode, st.mean, st.rstd, gam, et, st.xlo, st.xhi);
-      int8_t* dst = codes + warp * stride + (int64_t)g * Kg;
-      row_store_codes<TX>(seg, ni, lane, map, dst);
-      __syncwarp();
-      int cs = 0;
-      for (int i = 0; i < ni; ++i) {
-        const uint2 c = *reinterpret_cast<const uint2*>(dst + (size_t)(lane + 32 * i) * 8);
-        cs = __dp4a((int)c.x, 0x01010101, cs);
-        cs = __dp4a((int)c.y, 0x01010101, cs);
-      }
-      cs = warp_sum(cs);
-      if (lane == 0) { sh.csum[warp][g] = cs; sh.gamma[warp][g] = (float)gam; sh.eta[warp][g] = (float)et; }
     }
   }
   __syncthreads();
 
-  // 3. rows.  Lanes of absent tokens read zeros.
+  // ---- 3. rows.  Lanes of absent tokens read zeros.
   const bool tok_ok = g8 < a.M;
   const unsigned char* brow = tok_ok ? reinterpret_cast<const unsigned char*>(codes) + g8 * stride : smem;
   const uint32_t bmask = tok_ok ? 0xFFFFFFFFu : (uint32_t)(kZeroBytes - 1);
   const bool correct = a.eta_correction != 0;
   TY* y = reinterpret_cast<TY*>(a.y);
-  float out[4] = {0.f, 0.f, 0.f, 0.f};
-  int acc[8][4];
-  while (valid(cur)) {
-    const Item nn = next(nxt);
-    const int64_t r0 = cur.tile * kTileRows;
-    const int g = cur.t / nbg;
-    const int b0 = first_block(cur), nb = num_blocks(cur);
-    if (cur.t % nbg == 0) {                                    // a group starts
+  Item it3 = next(it2);
+  for (int64_t tile = tile0; tile < tiles; tile += tile_step) {
+    const int64_t r0 = tile * kTileRows;
+    float out[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int g = 0; g < a.G; ++g) {
+      int acc[8][4];
 #pragma unroll
-      for (int j = 0; j < 8; ++j)
+      for (int jj = 0; jj < 8; ++jj)
 #pragma unroll
-        for (int c = 0; c < 4; ++c) acc[j][c] = 0;
-    }
+        for (int c = 0; c < 4; ++c) acc[jj][c] = 0;
+      for (int b = 0; b < nbg; ++b) {
+        const int b0 = g * bpg + my_first + b * kPreload;
+        const int left = my_blocks - b * kPreload;
+        const int nb = left < kPreload ? left : kPreload;
 #pragma unroll
-    for (int i = 0; i < kPreload; ++i) {
-      if (i < nb) {
-        // B operand: the 8 planes' words for word qd (x0, x1) and word 4 + qd (x2, x3) of block b0 + i
-        const uint32_t off0 = (uint32_t)(32 * (8 * (b0 + i) + qd)) & bmask;
-        const uint32_t off1 = (uint32_t)(32 * (8 * (b0 + i) + 4 + qd)) & bmask;
-        const uint4 x0 = *reinterpret_cast<const uint4*>(brow + off0);
-        const uint4 x1 = *reinterpret_cast<const uint4*>(brow + off0 + 16);
-        const uint4 x2 = *reinterpret_cast<const uint4*>(brow + off1);
-        const uint4 x3 = *reinterpret_cast<const uint4*>(brow + off1 + 16);
-        const uint32_t bl[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-        const uint32_t bh[8] = {x2.x, x2.y, x2.z, x2.w, x3.x, x3.y, x3.z, x3.w};
+        for (int i = 0; i < kPreload; ++i) {
+          if (i < nb) {
+            // B operand: the 8 planes' words for word qd (x0, x1) and word 4 + qd (x2, x3) of block b0 + i
+            const uint32_t off0 = (uint32_t)(32 * (8 * (b0 + i) + qd)) & bmask;
+            const uint32_t off1 = (uint32_t)(32 * (8 * (b0 + i) + 4 + qd)) & bmask;
+            const uint4 x0 = *reinterpret_cast<const uint4*>(brow + off0);
+            const uint4 x1 = *reinterpret_cast<const uint4*>(brow + off0 + 16);
+            const uint4 x2 = *reinterpret_cast<const uint4*>(brow + off1);
+            const uint4 x3 = *reinterpret_cast<const uint4*>(brow + off1 + 16);
+            const uint32_t bl[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+            const uint32_t bh[8] = {x2.x, x2.y, x2.z, x2.w, x3.x, x3.y, x3.z, x3.w};
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const uint32_t m = 0x01010101u << j;
-          const uint32_t af[4] = {wa[i][0] & m, wa[i][1] & m, wa[i][2] & m, wa[i][3] & m};
-          mma_s8s8(acc[j], af, bl[j], bh[j]);
+            for (int jj = 0; jj < 8; ++jj) {
+              const uint32_t m = 0x01010101u << jj;
+              const uint32_t af[4] = {wa[i][0] & m, wa[i][1] & m, wa[i][2] & m, wa[i][3] & m};
+              mma_s8s8(acc[jj], af, bl[jj], bh[jj]);
+            }
+          }
         }
+        // the next batch's weights move up; the one after it starts loading
+#pragma unroll
+        for (int i = 0; i < kPreload; ++i)
+#pragma unroll
+          for (int c = 0; c < 4; ++c) wa[i][c] = wb[i][c];
+        if (valid(it3)) load_item(it3, wb);
+        it3 = next(it3);
       }
-    }
-    // the next item's weights move up; the one after it starts loading
-#pragma unroll
-    for (int i = 0; i < kPreload; ++i)
-#pragma unroll
-      for (int c = 0; c < 4; ++c) wa[i][c] = wb[i][c];
-    if (valid(nn)) load_item(nn, wb);
-    if (cur.t % nbg == nbg - 1) {                              // the group is complete: fold and rescale
-      const float beta_g = a.beta[g];
+      // the group is complete in this warp's half: sums over the set bits, per (row, token) of the fragment
+      int s[4];
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
-        int s = 0;
+        int t = 0;
 #pragma unroll
-        for (int j = 0; j < 7; ++j) s += acc[j][c] >> j;
-        s -= acc[7][c] >> 7;                                   // plane 7's bytes are 0x80 = -128 as s8
-        const int tok = 2 * qd + (c & 1);
-        if (tok < a.M) {
-          const int dot = 2 * s - sh.csum[tok][g];
-          const int64_t n = r0 + g8 + 8 * (c >> 1);
-          out[c] += dequant_term(dot, beta_g, sh.gamma[tok][g], correct ? sh.eta[tok][g] : 0.f,
-                                 correct ? a.rowsum[n * a.G + g] : 0, correct);
+        for (int jj = 0; jj < 7; ++jj) t += acc[jj][c] >> jj;
+        s[c] = t - (acc[7][c] >> 7);                             // plane 7's bytes are 0x80 = -128 as s8
+      }
+      if (h == 1) *reinterpret_cast<int4*>(sh.handover[pair][lane]) = make_int4(s[0], s[1], s[2], s[3]);
+      bar_sync(1 + pair, 64);
+      if (h == 0) {
+        const int4 o = *reinterpret_cast<const int4*>(sh.handover[pair][lane]);
+        const int so[4] = {o.x, o.y, o.z, o.w};
+        const float beta_g = a.beta[g];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int tok = 2 * qd + (c & 1);
+          if (tok < a.M) {
+            const int dot = 2 * (s[c] + so[c]) - sh.csum[tok][g];
+            const int64_t n = r0 + g8 + 8 * (c >> 1);
+            out[c] += dequant_term(dot, beta_g, sh.gamma[tok][g], correct ? sh.eta[tok][g] : 0.f,
+                                   correct ? a.rowsum[n * a.G + g] : 0, correct);
+          }
         }
       }
+      bar_sync(1 + pair, 64);                                    // the hand-over slot may be rewritten
     }
-    if (cur.t == nbt - 1) {                                    // the tile is complete
+    if (h == 0) {
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         const int tok = 2 * qd + (c & 1);
         if (tok < a.M) y[(int64_t)tok * a.N + r0 + g8 + 8 * (c >> 1)] = out_cast<TY>(out[c]);
-        out[c] = 0.f;
       }
     }
-    cur = nxt; nxt = nn;
   }
 }
 
+inline size_t batch_smem(int64_t M, int64_t K, size_t xsz, bool stage) {
+  return kZeroBytes + (size_t)M * (size_t)(K + kRowPad) + (stage ? (size_t)M * (size_t)K * xsz : 0);
+}
+
 template <typename TX, typename TY>
-cudaError_t run2(const BatchArgs& a, cudaStream_t s) {
+cudaError_t run2(BatchArgs a, cudaStream_t s) {
   int dev = 0, sms = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
   const int64_t tiles = a.N / kTileRows;
   const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
-  const size_t smem = kZeroBytes + (size_t)kBatchWarps * kStageBytes + (size_t)a.M * (size_t)(a.K + kRowPad);
+  a.stage_tokens = batch_smem(a.M, a.K, sizeof(TX), true) <= kSmemBudget ? 1 : 0;
+  const size_t smem = batch_smem(a.M, a.K, sizeof(TX), a.stage_tokens != 0);
   if ((e = cudaFuncSetAttribute(gemv_batch_kernel<TX, TY>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) !=
       cudaSuccess)
     return e;
@@ -261,8 +339,7 @@ cudaError_t run1(const BatchArgs& a, bl_dtype yt, cudaStream_t s) {
 
 bool gemv_batch_supported(int64_t M, int64_t K, int64_t N, int G) {
   return M >= 1 && G >= 1 && K % kBlockK == 0 && (K / G) % kBlockK == 0 && N % kTileRows == 0 &&
-         kZeroBytes + (size_t)kBatchWarps * kStageBytes +
-                 (size_t)(M < kBatchTokens ? M : kBatchTokens) * (size_t)(K + kRowPad) <= 220 * 1024;
+         batch_smem(M < kBatchTokens ? M : kBatchTokens, K, 0, false) <= kSmemBudget;
 }
 
 // M tokens in launches of up to 8; later launches find the weights in L2.
@@ -275,6 +352,8 @@ cudaError_t launch_gemv_batch(const GemvArgs& g, int64_t M, cudaStream_t s) {
     a.K = g.K; a.N = g.N; a.G = g.G; a.mode = (int)g.mode; a.ln_eps = g.ln_eps; a.eta_correction = g.eta_correction;
     a.W_packed = g.W_packed; a.beta = g.beta; a.rowsum = g.rowsum;
     a.y = reinterpret_cast<char*>(g.y) + (size_t)m0 * (size_t)g.N * ysz;
+    a.stage_tokens = 0;
+    a.inv_kg = 1.0 / (double)(g.K / g.G);
     cudaError_t e = cudaErrorInvalidValue;
     switch (g.xt) {
       case BL_F32: e = run1<float>(a, g.yt, s); break;
