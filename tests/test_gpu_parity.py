@@ -167,6 +167,18 @@ def test_quant_act(M, K, G, dtype, mode, gran, outliers, relu):
     assert out["x_q"].abs().max().item() <= 127
 
 
+def test_quant_act_per_tensor_status_word_and_workspace_reuse():
+    # The per-tensor path keeps its status word in the workspace; reusing one (uninitialised)
+    # workspace for calls of different shapes must leave it clear and the results unchanged.
+    ws = torch.full((B.workspace_bytes(B.OP_QUANT_ACT, 4096, 1, 4096, 2),), 0xA5, dtype=torch.uint8, device=DEV)
+    for M, K, G, dtype in ((4096, 1024, 2, "bf16"), (300, 4096, 1, "f16"), (9, 8192, 1, "bf16"), (33, 1000, 5, "f32")):
+        x = synth.make_x(M, K, DT[dtype], seed=M + K, outliers=True).to(DEV)
+        a = B.quant_act(x, G=G, gran=B.PER_TENSOR, ws=ws)
+        assert B.ws_status(ws) == B.OK
+        b = B.quant_act(x, G=G, gran=B.PER_TENSOR)
+        assert torch.equal(a["x_q"], b["x_q"]) and torch.equal(a["gamma"], b["gamma"])
+
+
 def test_quant_act_ties_and_degenerate_rows():
     # LN skipped, gamma = 128 planted: scale is exactly 1, so the half-to-even ties are exact.
     vals = [0.5, 1.5, 2.5, 3.5, -0.5, -1.5, -2.5, -3.5, 126.5, -126.5, 127.5, 128.0, 0.0, 1.0, -1.0, 2.0]
