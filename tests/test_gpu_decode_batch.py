@@ -21,6 +21,8 @@ DT = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}
     (13, 2048, 160, 1, "f16", "absmax", False),      # two launches, ragged second batch of 5
     (5, 8192, 64, 1, "bf16", "absmax", False),       # K above two register batches of weights
     (2, 7168, 112, 7, "bf16", "eta", True),          # seven groups of 1024
+    (8, 16384, 48, 2, "f16", "absmax", False),       # tokens too long to stage in shared memory: read from L2
+    (7, 256, 32, 1, "f32", "absmax", False),         # one K block: the second warp of every pair has no work
 ])
 def test_gemv_decode_batch(M, K, N, G, dtype, mode, relu):
     x = synth.make_x(M, K, DT[dtype], seed=K + N + M, outliers=False, relu=relu)
