@@ -26,7 +26,7 @@ constexpr int kTileHalves = kBk * kPitch;
 constexpr int kAttnSmem = 2 * 2 * kTileHalves * (int)sizeof(__half);   // two stages of (K, V)
 
 __device__ __forceinline__ void mma_f16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
+  asm(
       "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
@@ -110,14 +110,19 @@ attention_causal_kernel(const __half* __restrict__ q, const __half* __restrict__
     // S = Q K^T for this warp's 16 rows x 64 keys
     float s[8][4];
 #pragma unroll
-    for (int nt = 0; nt < 8; ++nt) {
-      s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+    for (int nt = 0; nt < 8; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+    // k-steps outside, key blocks inside: consecutive MMAs write different accumulators
 #pragma unroll
-      for (int kp = 0; kp < 4; ++kp) {                            // two k-steps of 16 per ldmatrix
-        uint32_t b[4];
+    for (int kp = 0; kp < 4; ++kp) {                              // two k-steps of 16 per ldmatrix
+#pragma unroll
+      for (int nt = 0; nt < 8; nt += 2) {
+        uint32_t b[4], c[4];
         ldmatrix_x4(b, Ks + (nt * 8 + (lane & 7)) * kPitch + kp * 32 + (lane >> 3) * 8);
+        ldmatrix_x4(c, Ks + ((nt + 1) * 8 + (lane & 7)) * kPitch + kp * 32 + (lane >> 3) * 8);
         mma_f16(s[nt], aq[2 * kp], b[0], b[1]);
+        mma_f16(s[nt + 1], aq[2 * kp], c[0], c[1]);
         mma_f16(s[nt], aq[2 * kp + 1], b[2], b[3]);
+        mma_f16(s[nt + 1], aq[2 * kp + 1], c[2], c[3]);
       }
     }
     if (kb * kBk + kBk - 1 > wrow) {                             // the tile reaches past a row: mask later keys
@@ -156,13 +161,16 @@ attention_causal_kernel(const __half* __restrict__ q, const __half* __restrict__
     }
     // O += P V
 #pragma unroll
-    for (int dt = 0; dt < 16; ++dt) {
+    for (int kp = 0; kp < 2; ++kp) {                              // two key steps of 16 per ldmatrix
 #pragma unroll
-      for (int kp = 0; kp < 2; ++kp) {                            // two key steps of 16 per ldmatrix
-        uint32_t b[4];
+      for (int dt = 0; dt < 16; dt += 2) {
+        uint32_t b[4], c[4];
         ldmatrix_x4_trans(b, Vs + (kp * 32 + (lane >> 3) * 8 + (lane & 7)) * kPitch + dt * 8);
+        ldmatrix_x4_trans(c, Vs + (kp * 32 + (lane >> 3) * 8 + (lane & 7)) * kPitch + (dt + 1) * 8);
         mma_f16(acc[dt], ap[2 * kp], b[0], b[1]);
+        mma_f16(acc[dt + 1], ap[2 * kp], c[0], c[1]);
         mma_f16(acc[dt], ap[2 * kp + 1], b[2], b[3]);
+        mma_f16(acc[dt + 1], ap[2 * kp + 1], c[2], c[3]);
       }
     }
   }
