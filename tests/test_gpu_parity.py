@@ -179,6 +179,27 @@ def test_quant_act_per_tensor_status_word_and_workspace_reuse():
         assert torch.equal(a["x_q"], b["x_q"]) and torch.equal(a["gamma"], b["gamma"])
 
 
+def test_quant_act_per_tensor_from_two_streams():
+    # The one-kernel per-tensor path is a cooperative launch whose CTAs wait for one another; calls
+    # issued from two streams (each with its own workspace) must neither block one another nor mix.
+    xs = [synth.make_x(2048, 4096, torch.bfloat16, seed=i, outliers=True).to(DEV) for i in range(2)]
+    ref = [B.quant_act(x, gran=B.PER_TENSOR) for x in xs]
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream() for _ in range(2)]
+    wss = [torch.empty(B.workspace_bytes(B.OP_QUANT_ACT, 2048, 1, 4096, 1), dtype=torch.uint8, device=DEV)
+           for _ in range(2)]
+    outs = [dict(x_q=torch.empty_like(r["x_q"]), gamma=torch.empty_like(r["gamma"]), eta=torch.zeros_like(r["eta"]))
+            for r in ref]
+    for _ in range(50):
+        for i, st in enumerate(streams):
+            with torch.cuda.stream(st):
+                B.quant_act(xs[i], gran=B.PER_TENSOR, out=outs[i], ws=wss[i])
+    torch.cuda.synchronize()
+    for i in range(2):
+        assert B.ws_status(wss[i]) == B.OK
+        assert torch.equal(outs[i]["x_q"], ref[i]["x_q"]) and torch.equal(outs[i]["gamma"], ref[i]["gamma"])
+
+
 def test_quant_act_ties_and_degenerate_rows():
     # LN skipped, gamma = 128 planted: scale is exactly 1, so the half-to-even ties are exact.
     vals = [0.5, 1.5, 2.5, 3.5, -0.5, -1.5, -2.5, -3.5, 126.5, -126.5, 127.5, 128.0, 0.0, 1.0, -1.0, 2.0]
