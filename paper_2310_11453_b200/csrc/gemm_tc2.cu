@@ -14,8 +14,9 @@
 //   warp 0      TMA producer for this CTA's codes tile
 //   warp 1      rank 0: MMA issuer for the pair (one thread); idle in rank 1
 //   warp 2      tensor-memory allocation (both CTAs, cta_group::2)
-//   warps 4-7   epilogue
-//   warps 8-15  weight expanders: two groups of 4 warps, group e fills k-block e of every ring slot;
+//   warps 4-11  epilogue: warp w reads the tensor-memory lanes of its quarter (w % 4) and takes half
+//               of the tile's 256 columns (warps 4-7 the first 128, warps 8-11 the rest)
+//   warps 12-19 weight expanders: two groups of 4 warps, group e fills k-block e of every ring slot;
 //               thread u of a group owns row u of this CTA's 128-row half of the B tile
 // A ring slot holds two k-blocks (256 weights): the MMA issuer, whose serial work per barrier round
 // trip bounds the kernel, waits and commits once per slot and issues 8 MMAs in between.
@@ -23,7 +24,7 @@
 // tmem_full (accumulator complete; committed to both).  full (rank 0 only): one barrier per slot
 // collects the TMA bytes of both CTAs' codes tiles (rank 1's copies complete on rank 0's barrier:
 // cp.async.bulk.tensor.cta_group::2) and the expander warps of the pair, so the issuer waits once
-// per slot.  tmem_empty (rank 0) takes the 8 epilogue warps of the pair.  Remote arrivals are
+// per slot.  tmem_empty (rank 0) takes the 16 epilogue warps of the pair.  Remote arrivals are
 // mbarrier.arrive on the mapa address of rank 0's barrier.
 //
 // Every wait is bounded; a limit that runs out raises the CTA's abort flag, records
@@ -45,7 +46,9 @@ constexpr int kBK = 128;                 // weights per k-block (one 128-byte sw
 constexpr int kSub = 2;                  // k-blocks per ring slot: one barrier round trip per 256 weights
 constexpr int kSlots = 3;                // ring slots of kSub x (codes tile + weights half-tile)
 constexpr int kGroups = kSub;            // expander groups of 4 warps; group e fills k-block e of every slot
-constexpr int kExpandWarp0 = 8;
+constexpr int kExpandWarp0 = 12;
+constexpr int kEpiWarps = 8;             // two per lane quarter; with four, heavier epilogues (residual, ReLU)
+                                         // and short K left the MMAs waiting for a free accumulator
 constexpr int kThreads = (kExpandWarp0 + 4 * kGroups) * 32;
 constexpr int kEpiWarp0 = 4;
 constexpr int kABytes = kBM * kBK;       // 16 KB
@@ -175,7 +178,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&ctl->tmem_full[b]), 1);
-      mbar_init(smem_u32(&ctl->tmem_empty[b]), 8);
+      mbar_init(smem_u32(&ctl->tmem_empty[b]), 2 * kEpiWarps);
     }
     ctl->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -299,7 +302,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
       if (lane == 0) mbar_arrive_cluster(full0 + 8u * (uint32_t)slot);
       if (++slot == kSlots) { slot = 0; phase ^= 1u; }
     }
-  } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + 4) {
+  } else if (warp >= kEpiWarp0 && warp < kEpiWarp0 + kEpiWarps) {
     // ---------------------------------------------------------------- epilogue (own 128 tokens)
     const int q = warp & 3;                                  // lane quarter this warp may read
     const int row = q * 32 + lane;
@@ -326,8 +329,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
         }
         if (kMode == 1 || (kMode == 2 && a.beta_rows == 0)) beta_c = a.beta[g];
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * (uint32_t)kBN;
+        const int c_first = ((warp - kEpiWarp0) >> 2) * (kBN / 64);      // this warp's half of the columns
 #pragma unroll 1
-        for (int c = 0; c < kBN / 32; ++c) {
+        for (int c = c_first; c < c_first + kBN / 64; ++c) {
           const int64_t n0 = n_base + c * 32;
           // beta blocks are multiples of 32 output features: one value per chunk, fetched while the
           // accumulators travel from tensor memory
