@@ -396,9 +396,15 @@ rows_tensor_fused(const T* __restrict__ x, int64_t segments, int64_t K, int G, i
   __shared__ int counter1, counter2;
   __shared__ unsigned long long part_lo[BL_MAX_GROUPS], part_hi[BL_MAX_GROUPS];
   __shared__ double gam_s[BL_MAX_GROUPS], eta_s[BL_MAX_GROUPS];
+  __shared__ unsigned long long copy_bar[kRowWarps][2];        // one mbarrier per warp and slot
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   uint4* slots = reinterpret_cast<uint4*>(stage + (size_t)warp * 2 * kSlotBytes);
   if (threadIdx.x == 0) { counter1 = 0; counter2 = 0; }
+  if (lane == 0) {
+    for (int c = 0; c < 2; ++c)
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"((uint32_t)__cvta_generic_to_shared(&copy_bar[warp][c])));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
   if (threadIdx.x < BL_MAX_GROUPS) { part_lo[threadIdx.x] = ~0ull; part_hi[threadIdx.x] = 0ull; }
   __syncthreads();
   pdl_wait();
@@ -410,16 +416,50 @@ rows_tensor_fused(const T* __restrict__ x, int64_t segments, int64_t K, int G, i
   const int n_keep = n < 2 * kRowWarps ? n : 2 * kRowWarps;     // handed out statically, stay in the slots
   const int n_dyn = n - n_keep;                                 // drawn through the counters
   const int ni = Kg / 256;
-  const int nv = ni * RowTraits<T>::kVecPerChunk;               // 16-byte pieces per lane
-  auto issue = [&](int64_t seg, uint4* slot, uint64_t policy) {
-    if (seg >= 0) {
-      const uint4* src = reinterpret_cast<const uint4*>(x + (seg / G) * K + (seg % G) * (int64_t)Kg);
-#pragma unroll 4
-      for (int i = 0; i < nv; ++i) cp_async16(slot + lane + 32 * i, src + lane + 32 * i, policy);
-    }
-    cp_async_commit();
-  };
   auto slot_of = [&](int c) { return slots + c * (kSlotBytes / 16); };
+  // A segment travels as ONE bulk copy (issued by lane 0, completing on the slot's mbarrier): the 16
+  // per-lane cp.async it replaces cost the warp about 1000 clocks of issue per segment.
+  const uint32_t seg_bytes = (uint32_t)(Kg * sizeof(T));
+  auto issue = [&](int64_t seg, int c, uint64_t policy) {
+    if (seg >= 0 && lane == 0) {
+      const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&copy_bar[warp][c]);
+      const uint32_t dst = (uint32_t)__cvta_generic_to_shared(slot_of(c));
+      const T* src = x + (seg / G) * K + (seg % G) * (int64_t)Kg;
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the lanes' reads of the slot come first
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(seg_bytes) : "memory");
+      asm volatile(
+          "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+          ::"r"(dst), "l"(src), "r"(seg_bytes), "r"(bar), "l"(policy) : "memory");
+    }
+  };
+  // Waits (with a limit) for the copy into slot c; a limit that runs out is recorded in the status
+  // word and the kernel goes on (its outputs are then undefined), so nothing can hang.
+  uint32_t parity = 0;                                           // bit c: phase of slot c's barrier to wait for
+  auto arrived = [&](int c) {
+    const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&copy_bar[warp][c]);
+    const uint32_t ph = (parity >> c) & 1u;
+    auto poll = [&]() {
+      uint32_t ok;
+      asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                   : "=r"(ok) : "r"(bar), "r"(ph) : "memory");
+      return ok != 0;
+    };
+    bool ok = poll();
+    if (!ok) {
+      unsigned long long t0;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+      for (unsigned it = 0; it < kMeetSpins && !ok; ++it) {
+        ok = poll();
+        if (!ok && (it & 255u) == 255u) {
+          unsigned long long now;
+          asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+          if (now - t0 > kMeetNs) break;
+        }
+      }
+      if (!ok && lane == 0) atomicExch(status, (uint32_t)BL_ERR_TIMEOUT);
+    }
+    parity ^= 1u << c;
+  };
 
   // ---- pass 1
   bool dyn_done = n_dyn == 0;
@@ -439,14 +479,13 @@ rows_tensor_fused(const T* __restrict__ x, int64_t segments, int64_t K, int G, i
   const uint64_t keep = l2_policy(true), last_use = l2_policy(false);
   int cur = 0;
   int64_t seg = draw1();
-  issue(seg, slot_of(0), keep);
+  issue(seg, 0, keep);
   int64_t seg_last = -1, seg_prev = -1;
   RowStats st_last = {0.0, 0.0, 0.f, 0.f}, st_prev = st_last;
   while (seg >= 0) {
     const int64_t next = draw1();
-    issue(next, slot_of(cur ^ 1), next >= rg.begin + n_dyn ? last_use : keep);
-    cp_async_wait_but_newest();
-    __syncwarp();
+    issue(next, cur ^ 1, next >= rg.begin + n_dyn ? last_use : keep);
+    arrived(cur);
     const RowStats st = row_stats<T>(slot_of(cur), ni, lane, ln_eps, inv_kg);
     if (lane == 0) {
       const int g = (int)(seg % G);
@@ -528,20 +567,18 @@ rows_tensor_fused(const T* __restrict__ x, int64_t segments, int64_t K, int G, i
   if (kept >= 1) code(seg_last, st_last, slot_of(cur));
   __syncwarp();
   seg = n_dyn > 0 ? draw2() : -1;
-  issue(seg, slot_of(cur), last_use);                            // overlaps the second retained segment
+  issue(seg, cur, last_use);                                     // overlaps the second retained segment
   if (kept >= 2) code(seg_prev, st_prev, slot_of(cur ^ 1));
   __syncwarp();
   while (seg >= 0) {
     const int64_t next = draw2();
-    issue(next, slot_of(cur ^ 1), last_use);
+    issue(next, cur ^ 1, last_use);
     const SegRecord rec = recs[seg];
-    cp_async_wait_but_newest();
-    __syncwarp();
+    arrived(cur);
     code(seg, RowStats{rec.mean, rec.rstd, rec.xlo, rec.xhi}, slot_of(cur));
     __syncwarp();
     seg = next; cur ^= 1;
   }
-  asm volatile("cp.async.wait_all;" ::: "memory");
 }
 
 // Unique, never zero, per call: high half drawn once per process, low half a call counter.
