@@ -117,7 +117,10 @@ bl_status bitlinear_binarize_pack(const void* W, bl_dtype wt, int64_t N, int64_t
  * PER_TENSOR is two (statistics, then codes).  For segments of up to 8 KB that are a multiple of
  * 256 features both passes run in one cooperative kernel whose CTAs wait for one another between
  * the passes, with a limit: after a PER_TENSOR call bitlinear_ws_status(ws, stream) reports
- * BL_ERR_TIMEOUT if that wait expired (codes are then not written).  Workspace: BL_OP_QUANT_ACT. */
+ * BL_ERR_TIMEOUT if that wait expired (codes are then not written).  Workspace: BL_OP_QUANT_ACT.
+ * PER_TOKEN needs no workspace (ws may be NULL).  Given one of at least 256 bytes, its first word
+ * becomes the call's status word and segments of the shape above are fetched with bulk copies whose
+ * bounded wait reports there (bitlinear_ws_status as above); the values written are the same. */
 bl_status bitlinear_quant_act(const void* x, bl_dtype xt, int64_t M, int64_t K, int G, int b,
                               bl_quant_mode mode, bl_gran gran, float ln_eps, int8_t* x_q,
                               float* gamma, float* eta, void* ws, size_t ws_bytes, void* stream);
@@ -287,7 +290,8 @@ bl_status bitlinear_attention_causal(const void* q, const void* k, const void* v
  * [T, 3d] buffer (k = q + d, v = q + 2d, ld_qkv = 3d); otherwise as three GEMMs.  The values
  * written are the same either way.  9 launches in the fused layout, 11 otherwise.
  * Workspace: BL_OP_BLOCK_FORWARD (codes, gamma, eta, quant and GEMM scratch).  Asynchronous on
- * `stream`; bitlinear_ws_status(ws, stream) reports a device-side timeout of the GEMMs. */
+ * `stream`; bitlinear_ws_status(ws, stream) reports a device-side timeout of any of the block's
+ * kernels (the first one clears the status word, the later ones only ever set it). */
 typedef struct {
   const uint8_t *W_q, *W_k, *W_v, *W_o, *W_up, *W_down;
   const float *beta_q, *beta_k, *beta_v, *beta_o, *beta_up, *beta_down;

@@ -188,7 +188,8 @@ def binarize_pack_nsplit(W, NB, G=1, layout=CANONICAL, alpha_in=None, want_rowsu
 
 
 def quant_act(x, G=1, mode=ABSMAX, gran=PER_TOKEN, ln_eps=1e-5, b=8, out=None, ws=None):
-    """bitlinear_quant_act.  x [M,K].  Returns dict(x_q i8 [M,K], gamma, eta f32)."""
+    """bitlinear_quant_act.  x [M,K].  Returns dict(x_q i8 [M,K], gamma, eta f32).
+    ws=False passes no workspace at all (allowed for PER_TOKEN only)."""
     M, K = x.shape
     dev = x.device
     out = dict(out or {})
@@ -199,9 +200,13 @@ def quant_act(x, G=1, mode=ABSMAX, gran=PER_TOKEN, ln_eps=1e-5, b=8, out=None, w
     gamma = gamma if gamma is not None else torch.empty(ns, dtype=torch.float32, device=dev)
     eta = out.get("eta")
     eta = eta if eta is not None else torch.zeros(ns, dtype=torch.float32, device=dev)
-    ws = _ws(workspace_bytes(OP_QUANT_ACT, M, 1, K, G), dev, ws)
+    if ws is False:
+        ws_ptr, ws_bytes = None, 0
+    else:
+        ws = _ws(workspace_bytes(OP_QUANT_ACT, M, 1, K, G), dev, ws)
+        ws_ptr, ws_bytes = _ptr(ws), ws.numel()
     code = lib().bitlinear_quant_act(_ptr(x), _dt(x), M, K, G, b, mode, gran, float(ln_eps), _ptr(x_q),
-                                     _ptr(gamma), _ptr(eta), _ptr(ws), ws.numel(), _stream())
+                                     _ptr(gamma), _ptr(eta), ws_ptr, ws_bytes, _stream())
     _check(code, "bitlinear_quant_act")
     return dict(x_q=x_q, gamma=gamma, eta=eta)
 

@@ -174,6 +174,9 @@ bl_status bitlinear_quant_act(const void* x, bl_dtype xt, int64_t M, int64_t K, 
     if (!aligned16(ws)) return BL_ERR_ALIGN;
   }
   QuantArgs a{x, xt, M, K, G, mode, gran, ln_eps, x_q, gamma, eta, ws};
+  // per-token scope needs no workspace; given one, its first word serves as the status word and the
+  // kernel may then use copies whose wait is bounded and reported there
+  if (gran == BL_PER_TOKEN && ws && ws_bytes >= kStatusBytes && aligned16(ws)) a.status = reinterpret_cast<uint32_t*>(ws);
   return launch_quant_act(a, (cudaStream_t)stream) == cudaSuccess ? BL_OK : BL_ERR_CUDA;
 }
 
@@ -296,12 +299,12 @@ bl_status bitlinear_forward(const void* x, bl_dtype xt, int64_t M, int64_t K, in
   float* gamma = reinterpret_cast<float*>(base + w.gamma);
   float* eta = reinterpret_cast<float*>(base + w.eta);
   QuantArgs q{x, xt, M, K, G, mode, gran, ln_eps, codes, gamma, eta, base + w.quant};
-  // One status word for the call: the per-tensor quant kernels clear it (and may report a timeout
-  // of their own), so the GEMM that follows must not clear it again.
+  // One status word for the call: the quant kernels clear it (and may report a timeout of their
+  // own), so the GEMM that follows must not clear it again.
   q.status = reinterpret_cast<uint32_t*>(base + w.status);
   if (launch_quant_act(q, s) != cudaSuccess) return BL_ERR_CUDA;
   GemmArgs a{};
-  a.keep_status = gran == BL_PER_TENSOR ? 1 : 0;
+  a.keep_status = 1;
   a.x_q = codes; a.M = M; a.K = K; a.N = N; a.G = G; a.W_packed = W_packed; a.acc = nullptr;
   a.y = y; a.yt = yt; a.beta = beta; a.gamma = gamma; a.eta = eta; a.gran = gran;
   a.rowsum = rowsum; a.eta_correction = eta_correction ? 1 : 0;
@@ -413,8 +416,14 @@ bl_status bitlinear_block_forward(const void* x, int batch, int seq, int heads, 
   float* eta = reinterpret_cast<float*>(base + c.eta);
 
   // LN + per-token quantisation of `in` [T,K] (fp16), then W~ x~ rescaled into `out` [T,N] (fp16).
+  // One status word for the whole block: the first kernel clears it, every later one keeps it.
+  uint32_t* status = reinterpret_cast<uint32_t*>(base + c.gemm);
+  bool first_kernel = true;
   auto quant = [&](const void* in, int64_t K, bl_quant_mode mode) -> bool {
     QuantArgs q{in, BL_F16, T, K, 1, mode, BL_PER_TOKEN, ln_eps, codes, gamma, eta, nullptr};
+    q.status = status;
+    q.keep_status = first_kernel ? 0 : 1;
+    first_kernel = false;
     return launch_quant_act(q, s) == cudaSuccess;
   };
   // out [T,N] (row stride ld) = [relu] BitLinear(codes) [+ res]; beta holds one entry per beta_rows features.
@@ -424,7 +433,7 @@ bl_status bitlinear_block_forward(const void* x, int batch, int seq, int heads, 
     g.x_q = codes; g.M = T; g.K = K; g.N = N; g.G = 1; g.W_packed = W; g.acc = nullptr; g.y = out; g.yt = BL_F16;
     g.beta = beta; g.gamma = gamma; g.eta = eta; g.gran = BL_PER_TOKEN; g.rowsum = nullptr; g.eta_correction = 0;
     g.beta_rows = beta_rows; g.relu = relu ? 1 : 0; g.residual = res; g.ld_res = d; g.ld_y = ld;
-    g.status = reinterpret_cast<uint32_t*>(base + c.gemm);
+    g.status = status; g.keep_status = 1;
     g.scratch = base + c.gemm + kStatusBytes;
     return launch_gemm_tc(g, s) == cudaSuccess;
   };

@@ -145,8 +145,10 @@ cudaError_t launch_binarize_pack(const PackArgs& a, cudaStream_t s);
 struct QuantArgs {
   const void* x; bl_dtype xt; int64_t M, K; int G; bl_quant_mode mode; bl_gran gran; float ln_eps;
   int8_t* x_q; float* gamma; float* eta; void* ws;
-  uint32_t* status = nullptr;                      // word for a device-side timeout (per-tensor scope);
-                                                   // nullptr: the first word of ws
+  uint32_t* status = nullptr;                      // word for a device-side timeout.  nullptr: per-tensor
+                                                   // scope uses the first word of ws, per-token scope runs
+                                                   // without bounded waits (per-lane copies)
+  int keep_status = 0;                             // an earlier kernel of the call already cleared the word
 };
 size_t quant_ws_bytes(int64_t M, int G);
 cudaError_t launch_quant_act(const QuantArgs& a, cudaStream_t s);

@@ -88,9 +88,9 @@ quant_per_token(const T* __restrict__ x, int64_t K, int G, int mode, float ln_ep
   }
 }
 
-__global__ void init_scope(TensorScope* sc, uint32_t* status) {
+__global__ void init_scope(TensorScope* sc, uint32_t* status, int clear_status) {
   const int g = threadIdx.x;
-  if (g == 0) *status = 0u;                          // these kernels have no device-side wait
+  if (g == 0 && clear_status) *status = 0u;                          // these kernels have no device-side wait
   if (g < BL_MAX_GROUPS) { sc->enc_min[g] = ~0ull; sc->enc_max[g] = 0ull; }
 }
 
@@ -192,25 +192,106 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 // lanes' pieces visible too.
 __device__ __forceinline__ void cp_async_wait_but_newest() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 
-// Draws the warp's next segment (-1 when the CTA's range is used up), starts its copy into
-// `slot` and closes the copy group (an empty one when there is nothing left to copy).
+// ---- bulk copies ---------------------------------------------------------------------------------------
+// With a status word to report through, a segment travels as ONE bulk copy issued by lane 0 and
+// completing on an mbarrier of the warp's slot: the 16 (or 32) cp.async per lane it replaces cost a
+// warp about 1000 clocks of issue per 8 KB.  The wait for it is bounded; a limit that runs out is
+// recorded in the status word and the kernel goes on (its outputs are then undefined), so nothing
+// can hang.  Without a status word the per-lane copies are used: their wait is not a spin loop.
+constexpr unsigned kMeetSpins = 1u << 22;                     // polls of a barrier or of the arrival tags
+constexpr unsigned long long kMeetNs = 2000000000ull;         // and a 2 s limit on the clock
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+// One lane, after the warp has finished reading dst.  bytes is a multiple of 16.
+__device__ __forceinline__ void bulk_issue(void* dst, const void* src, uint32_t bytes, unsigned long long* bar,
+                                           uint64_t policy) {
+  const uint32_t b = smem_u32(bar);
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the lanes' reads of the slot come first
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"(bytes) : "memory");
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+      ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(b), "l"(policy) : "memory");
+}
+// Waits for phase `ph` of the barrier; false when the limit ran out first.
+__device__ __forceinline__ bool bulk_wait(unsigned long long* bar, uint32_t ph) {
+  const uint32_t b = smem_u32(bar);
+  auto poll = [&]() {
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(b), "r"(ph) : "memory");
+    return ok != 0;
+  };
+  bool ok = poll();
+  if (!ok) {
+    unsigned long long t0;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    for (unsigned it = 0; it < kMeetSpins && !ok; ++it) {
+      ok = poll();
+      if (!ok && (it & 255u) == 255u) {
+        unsigned long long now;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+        if (now - t0 > kMeetNs) break;
+      }
+    }
+  }
+  return ok;
+}
+
+// A warp's staging area: 16 KB of shared memory (two slots, or one long one) and one mbarrier per slot.
+struct Staging {
+  uint4* slots;
+  unsigned long long* bars;
+  uint32_t* status;                                              // nullptr: per-lane cp.async
+  uint32_t parity;                                               // bit c: phase of slot c's barrier to wait for
+  __device__ __forceinline__ uint4* slot(int c) const { return slots + c * (kSlotBytes / 16); }
+};
+// Called by every thread before the kernel's first block barrier.
+__device__ __forceinline__ Staging staging_init(unsigned char* stage, unsigned long long (*bars)[2], uint32_t* status) {
+  const int warp = threadIdx.x >> 5;
+  Staging sg{reinterpret_cast<uint4*>(stage + (size_t)warp * 2 * kSlotBytes), bars[warp], status, 0u};
+  if ((threadIdx.x & 31) == 0) {
+    for (int c = 0; c < 2; ++c) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bars[warp][c])));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  return sg;
+}
+__device__ __forceinline__ void staging_wait(Staging& sg, int c, bool newest_pending, int lane) {
+  if (sg.status) {
+    if (!bulk_wait(&sg.bars[c], (sg.parity >> c) & 1u) && lane == 0) atomicExch(sg.status, (uint32_t)BL_ERR_TIMEOUT);
+    sg.parity ^= 1u << c;
+  } else if (newest_pending) {
+    cp_async_wait_but_newest();
+  } else {
+    asm volatile("cp.async.wait_all;" ::: "memory");
+  }
+  __syncwarp();
+}
+
+// Draws the warp's next segment (-1 when the CTA's range is used up) and starts its copy into
+// slot c (per-lane copies: also closes the copy group, an empty one when there is nothing left).
 // reverse walks the range from its end: the second per-tensor pass then begins with the rows the
 // first pass read last, the ones most likely still in L2.
 template <typename T>
 __device__ __forceinline__ int64_t stage_next(const T* __restrict__ x, const RowRange& rg, int64_t K, int G, int Kg,
-                                              bool reverse, uint64_t policy, int* counter, uint4* slot, int lane) {
+                                              bool reverse, uint64_t policy, int* counter, const Staging& sg, int c,
+                                              int lane) {
   int r = 0;
   if (lane == 0) r = atomicAdd(counter, 1);
   r = __shfl_sync(0xFFFFFFFFu, r, 0);
   int64_t seg = -1;
   if (rg.begin + r < rg.end) {
     seg = reverse ? rg.end - 1 - r : rg.begin + r;
-    const uint4* src = reinterpret_cast<const uint4*>(x + (seg / G) * K + (seg % G) * (int64_t)Kg);
-    const int nv = Kg / 256 * RowTraits<T>::kVecPerChunk;      // 16-byte pieces per lane
+    const T* src = x + (seg / G) * K + (seg % G) * (int64_t)Kg;
+    if (sg.status) {
+      if (lane == 0) bulk_issue(sg.slot(c), src, (uint32_t)(Kg * sizeof(T)), &sg.bars[c], policy);
+    } else {
+      const uint4* src16 = reinterpret_cast<const uint4*>(src);
+      const int nv = Kg / 256 * RowTraits<T>::kVecPerChunk;    // 16-byte pieces per lane
 #pragma unroll 4
-    for (int i = 0; i < nv; ++i) cp_async16(slot + lane + 32 * i, src + lane + 32 * i, policy);
+      for (int i = 0; i < nv; ++i) cp_async16(sg.slot(c) + lane + 32 * i, src16 + lane + 32 * i, policy);
+    }
   }
-  cp_async_commit();
+  if (!sg.status) cp_async_commit();
   return seg;
 }
 
@@ -218,10 +299,9 @@ __device__ __forceinline__ int64_t stage_next(const T* __restrict__ x, const Row
 // the next one already on its way.
 template <typename T, typename Body>
 __device__ __forceinline__ void for_each_segment(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg,
-                                                 bool reverse, uint64_t policy, int* counter, unsigned char* stage,
+                                                 bool reverse, uint64_t policy, int* counter, Staging& sg,
                                                  int64_t first_seg, Body body) {
   const int lane = threadIdx.x & 31;
-  uint4* slots = reinterpret_cast<uint4*>(stage + (size_t)(threadIdx.x >> 5) * 2 * kSlotBytes);
   const RowRange rg = cta_range(segments);
   // A segment of up to kSlotBytes leaves room for two slots (the next copy overlaps this body); a
   // longer one (up to 2 * kSlotBytes) fills the warp's whole area and its successor is copied after
@@ -231,43 +311,41 @@ __device__ __forceinline__ void for_each_segment(const T* __restrict__ x, int64_
   int64_t seg = first_seg;
   while (seg >= 0) {
     int64_t next = -1;
-    if (two_slots) {
-      next = stage_next<T>(x, rg, K, G, Kg, reverse, policy, counter, slots + (cur ^ 1) * (kSlotBytes / 16), lane);
-      cp_async_wait_but_newest();
-    } else {
-      asm volatile("cp.async.wait_all;" ::: "memory");
-    }
-    __syncwarp();
-    body(seg, slots + cur * (kSlotBytes / 16));
+    if (two_slots) next = stage_next<T>(x, rg, K, G, Kg, reverse, policy, counter, sg, cur ^ 1, lane);
+    staging_wait(sg, cur, two_slots, lane);
+    body(seg, sg.slot(cur));
     __syncwarp();                                    // every lane is done with the slot before it is refilled
     if (two_slots) cur ^= 1;
-    else next = stage_next<T>(x, rg, K, G, Kg, reverse, policy, counter, slots, lane);
+    else next = stage_next<T>(x, rg, K, G, Kg, reverse, policy, counter, sg, 0, lane);
     seg = next;
   }
 }
 // First draw of a warp (into slot 0), split off so that a kernel can put work between it and the loop.
 template <typename T>
 __device__ __forceinline__ int64_t first_segment(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg,
-                                                 bool reverse, uint64_t policy, int* counter, unsigned char* stage) {
-  uint4* slots = reinterpret_cast<uint4*>(stage + (size_t)(threadIdx.x >> 5) * 2 * kSlotBytes);
-  return stage_next<T>(x, cta_range(segments), K, G, Kg, reverse, policy, counter, slots, threadIdx.x & 31);
+                                                 bool reverse, uint64_t policy, int* counter, const Staging& sg) {
+  return stage_next<T>(x, cta_range(segments), K, G, Kg, reverse, policy, counter, sg, 0, threadIdx.x & 31);
 }
 
 template <typename T>
 __global__ void __launch_bounds__(kRowWarps * 32, 1)
 rows_per_token(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg, int mode, float ln_eps,
-               double inv_kg, int8_t* __restrict__ x_q, float* __restrict__ gamma, float* __restrict__ eta) {
+               double inv_kg, uint32_t* status, int clear_status, int8_t* __restrict__ x_q,
+               float* __restrict__ gamma, float* __restrict__ eta) {
   extern __shared__ __align__(16) unsigned char stage[];
   __shared__ int counter;
+  __shared__ unsigned long long copy_bar[kRowWarps][2];
   const int lane = threadIdx.x & 31;
   if (threadIdx.x == 0) counter = 0;
+  Staging sg = staging_init(stage, copy_bar, status);
   pdl_launch_dependents();
   __syncthreads();
   pdl_wait();
+  if (status && clear_status && blockIdx.x == 0 && threadIdx.x == 0) *status = 0u;   // a timeout comes seconds later
   const int ni = Kg / 256;
   const uint64_t pol = l2_policy(false);
-  const int64_t first = first_segment<T>(x, segments, K, G, Kg, false, pol, &counter, stage);
-  for_each_segment<T>(x, segments, K, G, Kg, false, pol, &counter, stage, first, [&](int64_t seg, const uint4* slot) {
+  const int64_t first = first_segment<T>(x, segments, K, G, Kg, false, pol, &counter, sg);
+  for_each_segment<T>(x, segments, K, G, Kg, false, pol, &counter, sg, first, [&](int64_t seg, const uint4* slot) {
     const RowStats st = row_stats<T>(slot, ni, lane, ln_eps, inv_kg);
     const double lo = ((double)st.xlo - st.mean) * st.rstd, hi = ((double)st.xhi - st.mean) * st.rstd;
     double gam, et;
@@ -287,23 +365,26 @@ rows_per_token(const T* __restrict__ x, int64_t segments, int64_t K, int G, int 
 template <typename T>
 __global__ void __launch_bounds__(kRowWarps * 32, 1)
 rows_tensor_stats(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg, float ln_eps, double inv_kg,
-                  ScopePartial* __restrict__ partials, SegRecord* __restrict__ recs, uint32_t* status) {
+                  ScopePartial* __restrict__ partials, SegRecord* __restrict__ recs, uint32_t* status,
+                  int clear_status) {
   extern __shared__ __align__(16) unsigned char stage[];
   __shared__ int counter;
   __shared__ unsigned long long part_lo[BL_MAX_GROUPS], part_hi[BL_MAX_GROUPS];
+  __shared__ unsigned long long copy_bar[kRowWarps][2];
   const int lane = threadIdx.x & 31;
   if (threadIdx.x == 0) counter = 0;
+  Staging sg = staging_init(stage, copy_bar, status);
   if (threadIdx.x < BL_MAX_GROUPS) { part_lo[threadIdx.x] = ~0ull; part_hi[threadIdx.x] = 0ull; }
   __syncthreads();
   pdl_wait();
   // Only now may the second pass be scheduled: its CTAs read x before their own wait, which is
   // safe because every CTA of this kernel has by then seen x complete.
   pdl_launch_dependents();
-  if (blockIdx.x == 0 && threadIdx.x == 0) *status = 0u;   // the two-kernel path has no device-side wait
+  if (clear_status && blockIdx.x == 0 && threadIdx.x == 0) *status = 0u;   // a timeout comes seconds later
   const int ni = Kg / 256;
   const uint64_t pol = l2_policy(true);                  // the second pass reads x again
-  const int64_t first = first_segment<T>(x, segments, K, G, Kg, false, pol, &counter, stage);
-  for_each_segment<T>(x, segments, K, G, Kg, false, pol, &counter, stage, first, [&](int64_t seg, const uint4* slot) {
+  const int64_t first = first_segment<T>(x, segments, K, G, Kg, false, pol, &counter, sg);
+  for_each_segment<T>(x, segments, K, G, Kg, false, pol, &counter, sg, first, [&](int64_t seg, const uint4* slot) {
     const RowStats st = row_stats<T>(slot, ni, lane, ln_eps, inv_kg);
     if (lane == 0) {
       const int g = (int)(seg % G);
@@ -322,20 +403,22 @@ rows_tensor_stats(const T* __restrict__ x, int64_t segments, int64_t K, int G, i
 template <typename T>
 __global__ void __launch_bounds__(kRowWarps * 32, 1)
 rows_tensor_codes(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg, int mode, int stat_ctas,
-                  const ScopePartial* __restrict__ partials, const SegRecord* __restrict__ recs,
+                  const ScopePartial* __restrict__ partials, const SegRecord* __restrict__ recs, uint32_t* status,
                   int8_t* __restrict__ x_q, float* __restrict__ gamma, float* __restrict__ eta) {
   extern __shared__ __align__(16) unsigned char stage[];
   __shared__ int counter;
   __shared__ double gam_s[BL_MAX_GROUPS], eta_s[BL_MAX_GROUPS];
+  __shared__ unsigned long long copy_bar[kRowWarps][2];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   if (threadIdx.x == 0) counter = 0;
+  Staging sg = staging_init(stage, copy_bar, status);
   pdl_launch_dependents();
   __syncthreads();
   const int ni = Kg / 256;
   const uint64_t pol = l2_policy(false);
   // x was complete before the first pass let this kernel be scheduled (see there), so the first
   // copies start before the wait for the first pass's records and extremes.
-  const int64_t first = first_segment<T>(x, segments, K, G, Kg, true, pol, &counter, stage);
+  const int64_t first = first_segment<T>(x, segments, K, G, Kg, true, pol, &counter, sg);
   pdl_wait();
   for (int g = warp; g < G; g += kRowWarps) {
     unsigned long long lo = ~0ull, hi = 0ull;
@@ -359,7 +442,7 @@ rows_tensor_codes(const T* __restrict__ x, int64_t segments, int64_t K, int G, i
     }
   }
   __syncthreads();
-  for_each_segment<T>(x, segments, K, G, Kg, true, pol, &counter, stage, first, [&](int64_t seg, const uint4* slot) {
+  for_each_segment<T>(x, segments, K, G, Kg, true, pol, &counter, sg, first, [&](int64_t seg, const uint4* slot) {
     const SegRecord rec = recs[seg];
     const int g = (int)(seg % G);
     const RowMap map = row_map(mode, rec.mean, rec.rstd, gam_s[g], eta_s[g], rec.xlo, rec.xhi);
@@ -383,83 +466,39 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
 __device__ __forceinline__ void st_release_u64(unsigned long long* p, unsigned long long v) {
   asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
-constexpr unsigned kMeetSpins = 1u << 22;                     // polls of the arrival tags before giving up
-constexpr unsigned long long kMeetNs = 2000000000ull;         // and a 2 s limit on the clock
 
 template <typename T>
 __global__ void __launch_bounds__(kRowWarps * 32, 1)
 rows_tensor_fused(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg, int mode, float ln_eps,
                   double inv_kg, ScopePartial* __restrict__ partials, SegRecord* __restrict__ recs,
                   unsigned long long* __restrict__ tags, unsigned long long tag, uint32_t* __restrict__ status,
-                  int8_t* __restrict__ x_q, float* __restrict__ gamma, float* __restrict__ eta) {
+                  int clear_status, int8_t* __restrict__ x_q, float* __restrict__ gamma, float* __restrict__ eta) {
   extern __shared__ __align__(16) unsigned char stage[];
   __shared__ int counter1, counter2;
   __shared__ unsigned long long part_lo[BL_MAX_GROUPS], part_hi[BL_MAX_GROUPS];
   __shared__ double gam_s[BL_MAX_GROUPS], eta_s[BL_MAX_GROUPS];
   __shared__ unsigned long long copy_bar[kRowWarps][2];        // one mbarrier per warp and slot
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  uint4* slots = reinterpret_cast<uint4*>(stage + (size_t)warp * 2 * kSlotBytes);
   if (threadIdx.x == 0) { counter1 = 0; counter2 = 0; }
-  if (lane == 0) {
-    for (int c = 0; c < 2; ++c)
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"((uint32_t)__cvta_generic_to_shared(&copy_bar[warp][c])));
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
+  Staging sg = staging_init(stage, copy_bar, status);
   if (threadIdx.x < BL_MAX_GROUPS) { part_lo[threadIdx.x] = ~0ull; part_hi[threadIdx.x] = 0ull; }
   __syncthreads();
   pdl_wait();
   pdl_launch_dependents();
-  if (blockIdx.x == 0 && threadIdx.x == 0) *status = 0u;        // a timeout (seconds later) overwrites it
+  if (clear_status && blockIdx.x == 0 && threadIdx.x == 0) *status = 0u;   // a timeout (seconds later) overwrites it
 
   const RowRange rg = cta_range(segments);
   const int n = (int)(rg.end - rg.begin);
   const int n_keep = n < 2 * kRowWarps ? n : 2 * kRowWarps;     // handed out statically, stay in the slots
   const int n_dyn = n - n_keep;                                 // drawn through the counters
   const int ni = Kg / 256;
-  auto slot_of = [&](int c) { return slots + c * (kSlotBytes / 16); };
-  // A segment travels as ONE bulk copy (issued by lane 0, completing on the slot's mbarrier): the 16
-  // per-lane cp.async it replaces cost the warp about 1000 clocks of issue per segment.
+  auto slot_of = [&](int c) { return sg.slot(c); };
   const uint32_t seg_bytes = (uint32_t)(Kg * sizeof(T));
   auto issue = [&](int64_t seg, int c, uint64_t policy) {
-    if (seg >= 0 && lane == 0) {
-      const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&copy_bar[warp][c]);
-      const uint32_t dst = (uint32_t)__cvta_generic_to_shared(slot_of(c));
-      const T* src = x + (seg / G) * K + (seg % G) * (int64_t)Kg;
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the lanes' reads of the slot come first
-      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(seg_bytes) : "memory");
-      asm volatile(
-          "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
-          ::"r"(dst), "l"(src), "r"(seg_bytes), "r"(bar), "l"(policy) : "memory");
-    }
+    if (seg >= 0 && lane == 0)
+      bulk_issue(sg.slot(c), x + (seg / G) * K + (seg % G) * (int64_t)Kg, seg_bytes, &sg.bars[c], policy);
   };
-  // Waits (with a limit) for the copy into slot c; a limit that runs out is recorded in the status
-  // word and the kernel goes on (its outputs are then undefined), so nothing can hang.
-  uint32_t parity = 0;                                           // bit c: phase of slot c's barrier to wait for
-  auto arrived = [&](int c) {
-    const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&copy_bar[warp][c]);
-    const uint32_t ph = (parity >> c) & 1u;
-    auto poll = [&]() {
-      uint32_t ok;
-      asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-                   : "=r"(ok) : "r"(bar), "r"(ph) : "memory");
-      return ok != 0;
-    };
-    bool ok = poll();
-    if (!ok) {
-      unsigned long long t0;
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
-      for (unsigned it = 0; it < kMeetSpins && !ok; ++it) {
-        ok = poll();
-        if (!ok && (it & 255u) == 255u) {
-          unsigned long long now;
-          asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
-          if (now - t0 > kMeetNs) break;
-        }
-      }
-      if (!ok && lane == 0) atomicExch(status, (uint32_t)BL_ERR_TIMEOUT);
-    }
-    parity ^= 1u << c;
-  };
+  auto arrived = [&](int c) { staging_wait(sg, c, false, lane); };
 
   // ---- pass 1
   bool dyn_done = n_dyn == 0;
@@ -629,14 +668,15 @@ cudaError_t launch_fused(const QuantArgs& a, cudaStream_t s, const T* x, int64_t
   static std::atomic<int> with_pdl{1};                          // dropped for good if the pair is refused once
   cfg.numAttrs = with_pdl.load() ? 2 : 1;
   const unsigned long long tag = next_tag();
+  const int clear = a.keep_status ? 0 : 1;
   e = cudaLaunchKernelEx(&cfg, kern, x, segments, a.K, a.G, Kg, (int)a.mode, a.ln_eps, inv_kg, partials, recs, tags,
-                         tag, status, a.x_q, a.gamma, a.eta);
+                         tag, status, clear, a.x_q, a.gamma, a.eta);
   if (e != cudaSuccess && cfg.numAttrs == 2) {
     (void)cudaGetLastError();
     with_pdl.store(0);
     cfg.numAttrs = 1;
     e = cudaLaunchKernelEx(&cfg, kern, x, segments, a.K, a.G, Kg, (int)a.mode, a.ln_eps, inv_kg, partials, recs, tags,
-                           tag, status, a.x_q, a.gamma, a.eta);
+                           tag, status, clear, a.x_q, a.gamma, a.eta);
   }
   return e;
 }
@@ -665,10 +705,11 @@ cudaError_t run_rows(const QuantArgs& a, cudaStream_t s) {
   cudaError_t e = rows_grid(segments, &grid);
   if (e != cudaSuccess) return e;
   const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
-  if (a.gran == BL_PER_TOKEN) {
+  const int clear = a.keep_status ? 0 : 1;
+  if (a.gran == BL_PER_TOKEN) {                                  // a.status may be nullptr: per-lane copies then
     if ((e = cudaFuncSetAttribute(rows_per_token<T>, attr, kRowStage)) != cudaSuccess) return e;
     return launch_pdl(rows_per_token<T>, grid, kThreads, kRowStage, s, x, segments, a.K, a.G, Kg, (int)a.mode,
-                      a.ln_eps, inv_kg, a.x_q, a.gamma, a.eta);
+                      a.ln_eps, inv_kg, a.status, clear, a.x_q, a.gamma, a.eta);
   }
   ScopePartial* partials = reinterpret_cast<ScopePartial*>(reinterpret_cast<char*>(a.ws) + kWsPartialOff);
   SegRecord* recs = reinterpret_cast<SegRecord*>(reinterpret_cast<char*>(a.ws) + kWsHeaderBytes);
@@ -681,10 +722,10 @@ cudaError_t run_rows(const QuantArgs& a, cudaStream_t s) {
   if ((e = cudaFuncSetAttribute(rows_tensor_stats<T>, attr, kRowStage)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(rows_tensor_codes<T>, attr, kRowStage)) != cudaSuccess) return e;
   e = launch_pdl(rows_tensor_stats<T>, grid, kThreads, kRowStage, s, x, segments, a.K, a.G, Kg, a.ln_eps, inv_kg,
-                 partials, recs, status);
+                 partials, recs, status, clear);
   if (e != cudaSuccess) return e;
   return launch_pdl(rows_tensor_codes<T>, grid, kThreads, kRowStage, s, x, segments, a.K, a.G, Kg, (int)a.mode,
-                    (int)grid, (const ScopePartial*)partials, (const SegRecord*)recs, a.x_q, a.gamma, a.eta);
+                    (int)grid, (const ScopePartial*)partials, (const SegRecord*)recs, status, a.x_q, a.gamma, a.eta);
 }
 
 template <typename T>
@@ -697,6 +738,8 @@ cudaError_t run(const QuantArgs& a, cudaStream_t s) {
   if (Kg % 256 == 0 && Kg <= RowTraits<T>::kMaxKg)               // whole chunks per lane, segment fits a slot
     return run_rows<T>(a, s);
   if (a.gran == BL_PER_TOKEN) {
+    // no device-side wait in this kernel: the word is only cleared for whoever reads it afterwards
+    if (a.status && !a.keep_status && (e = cudaMemsetAsync(a.status, 0, sizeof(uint32_t), s)) != cudaSuccess) return e;
     if (smem > 48 * 1024) {
       e = cudaFuncSetAttribute(quant_per_token<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e != cudaSuccess) return e;
@@ -711,7 +754,8 @@ cudaError_t run(const QuantArgs& a, cudaStream_t s) {
     e = cudaFuncSetAttribute(tensor_stats<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  init_scope<<<1, BL_MAX_GROUPS, 0, s>>>(sc, a.status ? a.status : reinterpret_cast<uint32_t*>(a.ws));
+  init_scope<<<1, BL_MAX_GROUPS, 0, s>>>(sc, a.status ? a.status : reinterpret_cast<uint32_t*>(a.ws),
+                                         a.keep_status ? 0 : 1);
   tensor_stats<T><<<grid, kQuantThreads, smem, s>>>(x, a.K, a.G, a.ln_eps, sc, recs);
   tensor_codes<T><<<grid, kQuantThreads, 0, s>>>(x, a.K, a.G, (int)a.mode, sc, recs, a.x_q, a.gamma, a.eta);
   return cudaGetLastError();

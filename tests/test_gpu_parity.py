@@ -165,6 +165,16 @@ def test_quant_act(M, K, G, dtype, mode, gran, outliers, relu):
         check_scalars(out["eta"].cpu().numpy(), ref["eta"])
         assert out["x_q"].min().item() >= 0
     assert out["x_q"].abs().max().item() <= 127
+    if gran == "token":
+        # With a workspace the segments arrive by bulk copies whose wait reports through its first
+        # word; without one, by per-lane copies.  Same values either way, and the word stays clear.
+        ws = torch.full((256,), 0xA5, dtype=torch.uint8, device=DEV)
+        with_ws = B.quant_act(x.to(DEV), G=G, mode=omode, gran=ogran, ln_eps=1e-5, ws=ws)
+        assert B.ws_status(ws) == B.OK                 # every per-token kernel clears (or leaves clear) the word
+        no_ws = B.quant_act(x.to(DEV), G=G, mode=omode, gran=ogran, ln_eps=1e-5, ws=False)
+        torch.cuda.synchronize()
+        for key in ("x_q", "gamma", "eta"):
+            assert torch.equal(out[key], with_ws[key]) and torch.equal(out[key], no_ws[key])
 
 
 def test_quant_act_per_tensor_status_word_and_workspace_reuse():
