@@ -39,13 +39,13 @@ constexpr int kBlockK = 256;             // weights per row and MMA step: 8 word
 constexpr int kPreload = 4;              // K blocks per batch; two batches are held in registers (2 x 4 x 4 words)
 constexpr int kRowPad = 16;              // bytes between token rows beyond K (bank spread of the B loads)
 constexpr int kZeroBytes = 64;           // zero area read by the lanes of absent tokens
-constexpr size_t kSmemBudget = 220 * 1024;
+constexpr size_t kSmemBudget = 210 * 1024;
 
 struct BatchShared {
   int csum[kBatchTokens][BL_MAX_GROUPS];
   float gamma[kBatchTokens][BL_MAX_GROUPS];
   float eta[kBatchTokens][BL_MAX_GROUPS];
-  double part_s[kBatchWarps], part_q[kBatchWarps];   // per-warp partial sums of one group segment
+  double part_s[kBatchWarps][32], part_q[kBatchWarps][32];   // per-warp, per-lane partial sums of one group segment
   float part_lo[kBatchWarps], part_hi[kBatchWarps];
   int part_c[kBatchWarps];
   int handover[kPairs][32][4];                       // second warp of a pair -> first, per group
@@ -161,28 +161,69 @@ gemv_batch_kernel(BatchArgs a) {
           pilot = 0.125f * (((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7])));
           if (a.ln_eps < 0.f) pilot = 0.f;
         }
-        float sum = 0.f, sq = 0.f, mn = INFINITY, mx = -INFINITY;
-        for (int rr = j; rr < rows_per_group; rr += P) {
-          Chunk<TX> ch; float v[8], d[8];
-          ch.load(seg, rr * 32 + lane); ch.unpack(v);
+        // The sums must not depend on how many warps share the token (a token's result is the same
+        // whatever else is in the batch), so their order of additions is fixed: chunk row rr belongs
+        // to strip rr % 16; a strip's sum is taken in fp32 per lane, rows ascending; the 16 strips
+        // are then added per lane in fp64 by halving (strip v with v + 8, then + 4, + 2, + 1), the
+        // first levels inside the warp that owns the strips, the rest across the token's warps;
+        // the lanes are added last.
+        float mn = INFINITY, mx = -INFINITY;
+        // this warp's strips: j, j + P, ... (at most 8); strip i >= 4 meets strip i - 4 as soon as it is done
+        double ls[kBatchWarps / 4], lq[kBatchWarps / 4];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) { d[i] = v[i] - pilot; mn = fminf(mn, v[i]); mx = fmaxf(mx, v[i]); }
-          sum += ((d[0] + d[1]) + (d[2] + d[3])) + ((d[4] + d[5]) + (d[6] + d[7]));
-          float p0 = d[0] * d[0], p1 = d[1] * d[1];
+        for (int i = 0; i < kBatchWarps / 2; ++i) {
+          float sum = 0.f, sq = 0.f;
+          if (i * P < kBatchWarps) {
+            for (int rr = j + i * P; rr < rows_per_group; rr += kBatchWarps) {
+              Chunk<TX> ch; float v[8], d[8];
+              ch.load(seg, rr * 32 + lane); ch.unpack(v);
 #pragma unroll
-          for (int i = 2; i < 8; i += 2) { p0 = fmaf(d[i], d[i], p0); p1 = fmaf(d[i + 1], d[i + 1], p1); }
-          sq += p0 + p1;
+              for (int e = 0; e < 8; ++e) { d[e] = v[e] - pilot; mn = fminf(mn, v[e]); mx = fmaxf(mx, v[e]); }
+              sum += ((d[0] + d[1]) + (d[2] + d[3])) + ((d[4] + d[5]) + (d[6] + d[7]));
+              float p0 = d[0] * d[0], p1 = d[1] * d[1];
+#pragma unroll
+              for (int e = 2; e < 8; e += 2) { p0 = fmaf(d[e], d[e], p0); p1 = fmaf(d[e + 1], d[e + 1], p1); }
+              sq += p0 + p1;
+            }
+          }
+          if (i < kBatchWarps / 4) { ls[i] = (double)sum; lq[i] = (double)sq; }   // strips it does not own: +0.0, exact
+          else if (i * P < kBatchWarps) { ls[i - kBatchWarps / 4] += (double)sum; lq[i - kBatchWarps / 4] += (double)sq; }
         }
-        const double S = warp_sum((double)sum), Q = warp_sum((double)sq);
+        {
+          // strips j + i P and j + (i + h) P differ by h P = 8, 4, 2 (only while h P < 16)
+          const int n = kBatchWarps / P;                         // strips of this warp: 1, 2, 4 or 8
+#pragma unroll
+          for (int h = kBatchWarps / 8; h >= 1; h >>= 1)
+            if (h < n) {
+#pragma unroll
+              for (int i = 0; i < kBatchWarps / 8; ++i)
+                if (i < h) { ls[i] += ls[i + h]; lq[i] += lq[i + h]; }
+            }
+        }
         mn = warp_min(mn); mx = warp_max(mx);
-        if (lane == 0) { sh.part_s[warp] = S; sh.part_q[warp] = Q; sh.part_lo[warp] = mn; sh.part_hi[warp] = mx; }
+        sh.part_s[warp][lane] = ls[0]; sh.part_q[warp][lane] = lq[0];
+        if (lane == 0) { sh.part_lo[warp] = mn; sh.part_hi[warp] = mx; }
         bar_sync(1 + tok, P * 32);
-        double St = 0.0, Qt = 0.0;
+        // across the token's warps, one quantity at a time (the kernel is at its register limit)
+        auto fold = [&](const double (*part)[32]) -> double {
+          double t[kBatchWarps / 2];
+#pragma unroll
+          for (int w = 0; w < kBatchWarps / 2; ++w) {
+            t[w] = w < P ? part[w0 + w][lane] : 0.0;
+            if (P > kBatchWarps / 2) t[w] += part[w0 + w + kBatchWarps / 2][lane];
+          }
+#pragma unroll
+          for (int h = kBatchWarps / 4; h >= 1; h >>= 1)
+            if (h < P) {
+#pragma unroll
+              for (int w = 0; w < kBatchWarps / 4; ++w)
+                if (w < h) t[w] += t[w + h];
+            }
+          return warp_sum(t[0]);
+        };
+        const double St = fold(sh.part_s), Qt = fold(sh.part_q);
         float xlo = INFINITY, xhi = -INFINITY;
-        for (int w = w0; w < w0 + P; ++w) {
-          St += sh.part_s[w]; Qt += sh.part_q[w];
-          xlo = fminf(xlo, sh.part_lo[w]); xhi = fmaxf(xhi, sh.part_hi[w]);
-        }
+        for (int w = w0; w < w0 + P; ++w) { xlo = fminf(xlo, sh.part_lo[w]); xhi = fmaxf(xhi, sh.part_hi[w]); }
         double mean = 0.0, rstd = 1.0;
         if (!(a.ln_eps < 0.f)) {
           const double dm = St * inv_kg;                      // mean - pilot

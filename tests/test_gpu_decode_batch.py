@@ -6,7 +6,7 @@ import torch
 from oracle import oracle as O
 from paper_2310_11453_b200 import binding as B
 from paper_2310_11453_b200 import synth
-from tests.test_gpu_parity import count_exact_ties
+from tests.test_gpu_parity import check_codes, count_exact_ties
 from tests.util import as_f32_np
 
 pytestmark = pytest.mark.gpu
@@ -39,8 +39,7 @@ def test_gemv_decode_batch(M, K, N, G, dtype, mode, relu):
     q = B.quant_act(xd, G=G, mode=omode, gran=B.PER_TOKEN, ln_eps=1e-5)
     ref_q = O.quant_act(as_f32_np(x), G=G, mode=omode, gran=O.PER_TOKEN, ln_eps=1e-5)
     codes = q["x_q"].cpu().numpy()
-    diff = codes.astype(np.int32) - ref_q["codes"].astype(np.int32)
-    assert np.abs(diff).max() <= 1 and np.count_nonzero(diff) <= max(4, 2e-4 * diff.size)
+    check_codes(codes, ref_q["codes"], x=as_f32_np(x), G=G, eta_per_token=(mode == "eta"))
     acc = O.matmul(codes, w_ref["bits"], G=G)
     for corr in ([False, True] if mode == "eta" else [False]):
         y = B.gemv_decode_batch(xd, w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode, ln_eps=1e-5,
@@ -56,7 +55,10 @@ def test_gemv_decode_batch(M, K, N, G, dtype, mode, relu):
         slack = ((max(1, int(1e-4 * K)) + ties) * step)[:, None]
         err = np.abs(y.cpu().numpy().astype(np.float64) - want)
         assert (err <= 1e-3 * rms + slack).all()
-        assert np.median(err) <= 1e-3 * rms                      # the typical element needs no slack
+        # the typical element needs no slack (an exact tie that went the other way moves every
+        # output of its token by one step, so tokens with such ties are left out)
+        if (ties == 0).any():
+            assert np.median(err[ties == 0]) <= 1e-3 * rms
     # 16-bit output is the rounding of the fp32 one
     y32 = B.gemv_decode_batch(xd, w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode, out_dtype=torch.float32)
     if dtype != "f32":
