@@ -3,9 +3,10 @@
 //
 // Two launches on the caller's stream, both HBM-bound (W is read twice: the means must be known
 // before any sign can be taken):
-//   1. reduce_partials  every block accumulates sum W and sum |W| of its rows: fp32 inside a
-//                       chunk of 8 weights, fp64 above; one (group, block) partial each - fixed
-//                       order, no atomics, so results are run-to-run identical;
+//   1. reduce_partials  every block accumulates sum W (every addition in fp64: alpha decides bits)
+//                       and sum |W| (fp32 inside a chunk of 8 weights, fp64 above) of its rows;
+//                       one (group, block) partial each - fixed order, no atomics, so results
+//                       are run-to-run identical;
 //   2. sign_pack        every CTA first folds the partials in the same fixed order (a few KB from
 //                       L2; this replaces a separate finalize launch), keeps per group the largest
 //                       float <= alpha_g (a float w exceeds the fp64 mean exactly when it exceeds
@@ -39,10 +40,13 @@ reduce_partials(const T* __restrict__ W, int64_t N, int64_t K, int G, PackWs* ws
       for (int64_t k = (int64_t)threadIdx.x * 8; k < Kg; k += (int64_t)kPackThreads * 8) {
         float v[8];
         Elem<T>::load8(row + k, v);
-        const float ps = ((v[0] + v[1]) + (v[2] + v[3])) + ((v[4] + v[5]) + (v[6] + v[7]));
+        // sum W decides bits (an element within the error of alpha of it would flip), so every
+        // addition is fp64; sum |W| only scales the output: fp32 inside the chunk is enough
+        const double ps = (((double)v[0] + (double)v[1]) + ((double)v[2] + (double)v[3])) +
+                          (((double)v[4] + (double)v[5]) + ((double)v[6] + (double)v[7]));
         const float pa = ((fabsf(v[0]) + fabsf(v[1])) + (fabsf(v[2]) + fabsf(v[3]))) +
                          ((fabsf(v[4]) + fabsf(v[5])) + (fabsf(v[6]) + fabsf(v[7])));
-        s += (double)ps;
+        s += ps;
         a += (double)pa;
       }
     }

@@ -132,4 +132,10 @@ def test_forward_latent_is_pack_then_forward(M, K, N, G, wdtype, mode, gran):
                     eta_correction=corr)
     rms = np.sqrt((ref["y"] ** 2).mean())
     err = np.abs(got["y"].cpu().numpy().astype(np.float64) - ref["y"])
-    assert np.median(err) <= 1e-3 * rms and np.quantile(err, 0.999) <= 2e-2 * rms
+    # one quantisation step of slack per code of the token that differs from the oracle's (rounding
+    # ties; the codes themselves are checked in the quantisation tests)
+    q = B.quant_act(x, G=G, mode=omode, gran=ogran)
+    flips = np.abs(q["x_q"].cpu().numpy().astype(np.int32) - ref["codes"].astype(np.int32)).sum(axis=1)
+    gam = ref["gamma"] if gran == "token" else np.broadcast_to(ref["gamma"], (M, G))
+    step = (w_ref["beta"][None, :] * gam / 128.0).max(axis=1)
+    assert (err <= 1e-3 * rms + (flips * step)[:, None]).all()
