@@ -18,6 +18,7 @@ import torch
 from oracle import oracle as O
 from paper_2310_11453_b200 import binding as B
 from paper_2310_11453_b200 import synth
+from tests.test_gpu_parity import check_codes
 from tests.util import as_f32_np
 
 pytestmark = pytest.mark.gpu
@@ -41,10 +42,8 @@ def check_bitlinear_stage(x_in, y_out, w_ref, mode, samples, seed):
     q_ref = O.quant_act(x, mode=omode, gran=O.PER_TOKEN, ln_eps=1e-5)
     q = B.quant_act(x_in, mode=omode, gran=B.PER_TOKEN, ln_eps=1e-5)
     codes = q["x_q"].cpu().numpy()
-    diff = codes.astype(np.int32) - q_ref["codes"].astype(np.int32)
-    assert np.abs(diff).max() <= 1
     # exact ties of the eta form (rational pre-rounding values) are valid either way; the rest is counted
-    assert np.count_nonzero(diff) <= max(4, 2e-4 * diff.size if mode == "eta" else 1e-4 * diff.size)
+    check_codes(codes, q_ref["codes"], x=x, G=1, eta_per_token=(mode == "eta"))
     rng = np.random.default_rng(seed)
     ms, ns = rng.integers(0, T, samples), rng.integers(0, N, samples)
     acc = O.matmul_samples(codes, w_ref["bits"], ms, ns)[:, 0].astype(np.float64)
@@ -75,6 +74,7 @@ def run_block(batch, seq, heads, ffn, seed, attn_rows, fused_qkv):
     # attention core on the GPU's q, k, v
     rows = np.unique(np.concatenate([[0, 1, 63, 64, seq - 1, T - seq, T - 1],
                                      np.random.default_rng(seed).integers(0, T, attn_rows)])).astype(np.int64)
+    rows = rows[rows < T]
     a_ref = O.attention_rows(as_f32_np(out["q"].contiguous()), as_f32_np(out["k"].contiguous()),
                              as_f32_np(out["v"].contiguous()), batch, seq, heads, 128, rows)
     a_gpu = out["a"].cpu().float().numpy()[rows].astype(np.float64)
