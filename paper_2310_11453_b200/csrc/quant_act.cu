@@ -152,16 +152,17 @@ tensor_codes(const T* __restrict__ x, int64_t K, int G, int mode, const TensorSc
 // on one, the asynchronous copies (cp.async, 16 bytes per lane and instruction) of its next
 // segment land in the other, so every warp keeps a segment's worth of HBM traffic outstanding
 // whatever it is computing.  A longer segment takes the whole area; its successor is copied after
-// the work on it, and the other eleven warps keep the memory system busy meanwhile.  Waiting is
+// the work on it, and the other warps keep the memory system busy meanwhile.  Waiting is
 // cp.async.wait_group: no barrier objects, no spin loops.  A warp walks its segment in chunks of
 // 8 elements per lane (a short rolled loop: small code, few registers), with warp shuffles for
 // the reductions and no block barrier inside the loop.  Sums are fp32 inside a lane and fp64
 // across lanes, in one pass over deviations from a pilot value.  Reciprocals and the inverse
 // square root are hardware seeds refined by Newton steps in fp64 (below one ulp of fp64 after two
 // steps), which keeps fp64 division and square-root routines out of the kernels.
-constexpr int kRowWarps = 12;
+constexpr int kRowWarps = 14;              // as many as shared memory holds: 14 x 16 KB of staging + 2.3 KB static
 constexpr int kSlotBytes = 8192;
 constexpr int kRowStage = kRowWarps * 2 * kSlotBytes;
+static_assert(kRowStage + 3 * 1024 <= 227 * 1024, "staging plus the kernels' static shared memory must fit one SM");
 template <typename T> struct RowTraits {                      // chunk = 8 consecutive elements
   static constexpr int kVecPerChunk = sizeof(T) == 4 ? 2 : 1; // 16-byte pieces per chunk
   static constexpr int kMaxKg = 2 * kSlotBytes / (int)sizeof(T);   // a warp's whole staging area
@@ -456,7 +457,7 @@ rows_tensor_codes(const T* __restrict__ x, int64_t segments, int64_t K, int G, i
 // statically: they are still in the warp's two slots when the pass ends.  Then the CTAs meet: each
 // publishes a tag (unique to the call, so the array needs no clearing) after its partial extremes,
 // and waits, with a limit, until all tags of the grid show it.  Pass 2 codes the retained segments
-// straight from shared memory (2 x 12 per SM that are not read from HBM again) and then the rest of
+// straight from shared memory (two per warp that are not read from HBM again) and then the rest of
 // its range backwards, as rows_tensor_codes does.
 __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
   unsigned long long v;
