@@ -201,7 +201,14 @@ def run_b200(args):
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K_steps)]
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    # The stream must not run dry at the start of the timed region: after the barrier the GPU is
+    # idle and the first steps would be timed with the host's launch latency inside them.  A fill
+    # of a buffer larger than L2 (which also leaves L2 cold) keeps the GPU busy while the host
+    # queues the first steps; t0 is recorded behind it.
+    head_start = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
     with ClockSampler(local) as clocks:
+        head_start.zero_()
+        head_start.zero_()
         t0.record()
         for i in range(K_steps):
             step(i, evs[i])
