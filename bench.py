@@ -352,6 +352,7 @@ def bench_decode(B, synth, dev, peaks):
         Wd = torch.randn((N, K), generator=gen, device=dev, dtype=torch.float32) * synth.W_STD
         packs.append(B.binarize_pack(Wd, layout=B.DECODE, want_rowsum=False))
         del Wd
+    torch.cuda.synchronize()                             # decode reads its weights ahead of stream order
     x = synth.make_x(calls, K, torch.float16, seed=1, outliers=False).to(dev)
     y = torch.empty((calls, N), dtype=torch.float16, device=dev)
 

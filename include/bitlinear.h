@@ -5,6 +5,9 @@
  *   step 1  LN(x) = (x - E x) / sqrt(Var x + eps)                         Eq. 12 (per group: Eq. 15)
  *   step 2  x~ = Clip(round(x^.Q_b/gamma), -(Q_b-1), Q_b-1), gamma = max|x^|   Eq. 4-5
  *           or Clip(round((x^-eta).Q_b/gamma), 0, Q_b-1), eta = min x^         Eq. 6
+ *           (in this form gamma = max x^ - min x^, the range of the shifted values: a departure
+ *           from Eq. 5 / 14 as printed, whose gamma = ||x||_inf would not map onto [0, Q_b];
+ *           the gamma returned for BL_ETA is this range)
  *   step 3  W~ = Sign(W - alpha), alpha = mean W, beta = mean|W|          Eq. 1-3, 12 (per group: Eq. 13)
  *   step 4  acc = W~ x~ in exact integers, rescaled by beta.gamma/Q_b     Eq. 7, 11
  * Symbols follow the paper: M tokens, K input features (the contraction and the group
@@ -13,10 +16,14 @@
  * Conventions that hold for every entry point unless it says otherwise
  *   - Every data pointer is a DEVICE pointer owned by the caller; matrices are dense row-major;
  *     base addresses are 16-byte aligned (BL_ERR_ALIGN otherwise).
- *   - The library allocates nothing and keeps no state between calls.  Scratch comes from the
+ *   - The library allocates nothing and keeps no results between calls.  Scratch comes from the
  *     caller as (ws, ws_bytes); ask bitlinear_workspace_bytes() for the size.  The workspace
  *     may be reused by the next call on the same stream; it holds nothing the caller needs
- *     except the status word read by bitlinear_ws_status().
+ *     except the status word read by bitlinear_ws_status().  What the library does hold, per
+ *     process: caches of device attributes and of per-kernel launch set-up (keyed by device
+ *     ordinal), a call counter that makes the arrival tags of the cooperative LN+quant kernel
+ *     unique, the setting of bitlinear_debug_wait_limit, and the fixed device array behind
+ *     bitlinear_quant_act_noalloc.  None of it changes a result.
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default
  *     stream) and never synchronise.
  *   - Errors are detected on the host before any launch and returned as a bl_status; nothing
@@ -242,7 +249,16 @@ bl_status bitlinear_binarize_pack_nsplit(const void* W, bl_dtype wt, int64_t N, 
 
 /* Steps 1, 2, 4 for one token (M = 1), fused in a single kernel that streams the packed
  * weights once; Eq. 11 with per-token gamma.  W_packed must be in DECODE layout.
- *   x [K] of dtype xt;  y [N] of dtype yt.  No workspace, no device-side waits. */
+ *   x [K] of dtype xt;  y [N] of dtype yt.  K % 256 == 0, K <= 32768, N % 16 == 0, and for G > 1
+ *   K_g % 128 == 0 (BL_ERR_SHAPE otherwise).  No workspace.
+ * The weights are constants of the model and are read AHEAD of stream order: the kernel starts
+ * copying W_packed into shared memory while earlier work on `stream` may still be running
+ * (programmatic dependent launch), so whatever wrote W_packed must have completed before this
+ * call is made (a pack on the same stream: synchronise once after packing).  x, beta, rowsum
+ * and y are only touched in stream order.
+ * The one device-side wait (for those copies) is bounded; if it ever ran out, the affected warps
+ * read their weights from global memory instead, so there is no status to collect and y is the
+ * same either way. */
 bl_status bitlinear_gemv_decode(const void* x, bl_dtype xt, int64_t K, int64_t N, int G, int b,
                                 bl_quant_mode mode, float ln_eps, int eta_correction,
                                 const uint8_t* W_packed, const float* beta,
@@ -307,6 +323,17 @@ bl_status bitlinear_block_forward(const void* x, int batch, int seq, int heads, 
 /* Synchronises `stream`, then reads the status word a previous bitlinear_forward or
  * bitlinear_matmul_i32 call left in `ws`.  BL_OK, BL_ERR_TIMEOUT, or BL_ERR_CUDA. */
 bl_status bitlinear_ws_status(const void* ws, void* stream);
+
+/* Test and diagnostic hook: caps the number of polls that the bounded device-side waits of
+ * kernels launched afterwards by this process may make (bitlinear_gemv_decode's wait for its
+ * weight copies; the meeting between the two passes of the cooperative per-tensor kernel of
+ * bitlinear_quant_act).  polls < 0 restores the built-in limits; 0 means a single poll.
+ * meet_skew != 0 additionally makes the cooperative kernel wait for an arrival tag that no CTA
+ * publishes, so that its wait runs out by construction: the kernel then records
+ * BL_ERR_TIMEOUT in the status word, writes no codes and returns (nothing hangs, traps or
+ * faults).  Process-wide and not synchronised with calls in flight on other host threads; not for
+ * production use.  Always returns BL_OK. */
+bl_status bitlinear_debug_wait_limit(int64_t polls, int meet_skew);
 
 #ifdef __cplusplus
 }

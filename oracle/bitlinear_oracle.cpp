@@ -5,13 +5,16 @@
 // notation.  It shares no code, header, table or constant with the CUDA library; only the
 // tests, the smoke check and the CPU-baseline leg of the benchmark may call it.
 //
-// Conventions fixed where the paper is silent (each is listed in the design notes):
+// Conventions fixed where the paper is silent, and one departure from it as printed:
 //   * rounding is round-half-to-even (nearbyint under FE_TONEAREST) applied to the double
 //     product, then the clip: codes lie in [-(Q_b-1), Q_b-1], or [0, Q_b-1] in eta mode;
 //   * Sign(0) = -1 (Eq. 2), evaluated on the double difference W_ij - alpha_g;
 //   * groups split the contraction dimension K into G equal slices (Eq. 13-15);
 //   * LN has no gain or bias and uses the population variance (Eq. 12);
-//   * gamma == 0 gives all-zero codes (no division by zero).
+//   * gamma == 0 gives all-zero codes (no division by zero);
+//   * in the eta form (Eq. 6) gamma = max x^ - min x^, the range of the shifted values.  This departs
+//     from Eq. 5 / 14 as printed, which define gamma = ||x||_inf once and redefine only eta for Eq. 6:
+//     with that gamma the shifted values would not land in [0, Q_b], which Eq. 6 says they do.
 //
 // Pins (tests/test_oracle_pins.py): hand-computed worked examples under tests/golden/,
 // closed forms for alpha/beta, the Sign tie, code bounds and saturation, the half-to-even

@@ -2,6 +2,11 @@
 // Nothing here allocates device memory or synchronises (bitlinear_ws_status excepted).
 #include "common.cuh"
 
+namespace bl {
+std::atomic<long long> g_debug_wait_polls{-1};
+std::atomic<int> g_debug_meet_skew{0};
+}  // namespace bl
+
 namespace {
 
 using namespace bl;
@@ -466,6 +471,12 @@ bl_status bitlinear_ws_status(const void* ws, void* stream) {
   if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return BL_ERR_CUDA;
   if (cudaMemcpy(&word, ws, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return BL_ERR_CUDA;
   return word == 0 ? BL_OK : BL_ERR_TIMEOUT;
+}
+
+bl_status bitlinear_debug_wait_limit(int64_t polls, int meet_skew) {
+  g_debug_wait_polls.store(polls < 0 ? -1 : (long long)polls, std::memory_order_relaxed);
+  g_debug_meet_skew.store(meet_skew ? 1 : 0, std::memory_order_relaxed);
+  return BL_OK;
 }
 
 }  // extern "C"

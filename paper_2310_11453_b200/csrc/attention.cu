@@ -187,31 +187,6 @@ attention_causal_kernel(const __half* __restrict__ q, const __half* __restrict__
   }
 }
 
-// y += r (residual), or y = max(y, 0): the block's elementwise glue, 8 halves per thread.
-__global__ void __launch_bounds__(256)
-add_inplace_kernel(__half* __restrict__ y, const __half* __restrict__ r, int64_t n8) {
-  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
-  if (i >= n8) return;
-  uint4 a = reinterpret_cast<uint4*>(y)[i];
-  const uint4 b = __ldg(reinterpret_cast<const uint4*>(r) + i);
-  __half2* pa = reinterpret_cast<__half2*>(&a);
-  const __half2* pb = reinterpret_cast<const __half2*>(&b);
-#pragma unroll
-  for (int j = 0; j < 4; ++j) pa[j] = __hadd2(pa[j], pb[j]);
-  reinterpret_cast<uint4*>(y)[i] = a;
-}
-__global__ void __launch_bounds__(256)
-relu_inplace_kernel(__half* __restrict__ y, int64_t n8) {
-  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
-  if (i >= n8) return;
-  uint4 a = reinterpret_cast<uint4*>(y)[i];
-  __half2* pa = reinterpret_cast<__half2*>(&a);
-  const __half2 z = __float2half2_rn(0.f);
-#pragma unroll
-  for (int j = 0; j < 4; ++j) pa[j] = __hmax2(pa[j], z);
-  reinterpret_cast<uint4*>(y)[i] = a;
-}
-
 }  // namespace
 
 cudaError_t launch_attention_causal(const void* q, const void* k, const void* v, void* o, int batch, int S,
@@ -223,19 +198,6 @@ cudaError_t launch_attention_causal(const void* q, const void* k, const void* v,
   attention_causal_kernel<<<grid, kAttnWarps * 32, kAttnSmem, s>>>(
       reinterpret_cast<const __half*>(q), reinterpret_cast<const __half*>(k), reinterpret_cast<const __half*>(v),
       reinterpret_cast<__half*>(o), S, ld, ld_o, scale_log2);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_add_inplace(void* y, const void* r, int64_t n, cudaStream_t s) {
-  const int64_t n8 = n / 8;
-  add_inplace_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, s>>>(reinterpret_cast<__half*>(y),
-                                                                  reinterpret_cast<const __half*>(r), n8);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_relu_inplace(void* y, int64_t n, cudaStream_t s) {
-  const int64_t n8 = n / 8;
-  relu_inplace_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, s>>>(reinterpret_cast<__half*>(y), n8);
   return cudaGetLastError();
 }
 

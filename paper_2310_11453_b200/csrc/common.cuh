@@ -7,9 +7,17 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/bitlinear.h"
 
 namespace bl {
+
+// Test hook behind bitlinear_debug_wait_limit (defined in api.cu, read by the launchers when a
+// call is made): cap on the polls of the bounded device-side waits (negative: built-in limits),
+// and whether the cooperative LN+quant kernel waits for a tag that nobody publishes.
+extern std::atomic<long long> g_debug_wait_polls;
+extern std::atomic<int> g_debug_meet_skew;
 
 // Programmatic dependent launch.  A kernel launched through launch_pdl() may be scheduled while
 // the kernel before it on the stream is still running: it calls pdl_wait() before its first
@@ -172,8 +180,7 @@ struct GemmArgs {
   void* scratch;                                   // gemm_tc_scratch_bytes(G) bytes (tensor-core path)
 };
 cudaError_t launch_gemm_simple(const GemmArgs& a, cudaStream_t s);
-cudaError_t launch_gemm_tc(const GemmArgs& a, cudaStream_t s);
-cudaError_t launch_gemm_tc2(const GemmArgs& a, cudaStream_t s);   // two SMs per tile
+cudaError_t launch_gemm_tc(const GemmArgs& a, cudaStream_t s);      // tcgen05, two SMs per tile (gemm_tc2.cu)
 bool gemm_tc_supported(int64_t M, int64_t K, int64_t N, int G);
 size_t gemm_tc_scratch_bytes(int64_t M, int64_t N, int G);   // host-only, no device query
 
@@ -187,11 +194,9 @@ cudaError_t launch_gemv_decode(const GemvArgs& a, cudaStream_t s);
 cudaError_t launch_gemv_batch(const GemvArgs& a, int64_t M, cudaStream_t s);
 bool gemv_batch_supported(int64_t M, int64_t K, int64_t N, int G);
 
-// Decoder-block glue (fp16): causal attention core and the elementwise steps.
+// Decoder-block glue (fp16): the causal attention core.
 cudaError_t launch_attention_causal(const void* q, const void* k, const void* v, void* o, int batch, int S,
                                     int heads, int64_t ld, int64_t ld_o, cudaStream_t s);
-cudaError_t launch_add_inplace(void* y, const void* r, int64_t n, cudaStream_t s);   // y += r, n % 8 == 0
-cudaError_t launch_relu_inplace(void* y, int64_t n, cudaStream_t s);                 // y = max(y, 0)
 
 // Host-side layout maps (also exported through bitlinear_layout_index).
 int64_t prefill_bytes(int64_t N, int64_t K);

@@ -30,6 +30,8 @@
 // Every wait is bounded; a limit that runs out raises the CTA's abort flag, records
 // BL_ERR_TIMEOUT and lets every role fall through to the common exit (cluster barrier, tensor
 // memory freed).  The partner then runs into its own limits.  No multicast loads are used.
+#include <atomic>
+
 #include "tc_common.cuh"
 
 namespace bl {
@@ -435,45 +437,55 @@ cudaError_t launch(const GemmArgs& a, cudaStream_t s) {
           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return cudaErrorInvalidValue;
-  static bool attr_set[3][3] = {};
   auto kern = gemm_tc2_kernel<kMode, TY>;
-  const int ti = kMode == 0 ? 0 : (int)a.yt;
-  if (!attr_set[kMode][ti]) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (e != cudaSuccess) return e;
-    attr_set[kMode][ti] = true;
-  }
   int dev = 0, sms = 148;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  // Per instantiation and device ordinal: 0 until the kernel's shared-memory size has been raised
+  // on that device, then the number of clusters that can be resident at once (the persistent grid
+  // never has more).  Devices beyond the table are set up on every call.
+  constexpr int kMaxDevices = 64;
+  static std::atomic<int> resident[kMaxDevices];
+  int cap = dev < kMaxDevices ? resident[dev].load(std::memory_order_acquire) : 0;
   const int64_t tiles = ((a.M + kPairM - 1) / kPairM) * ((a.N + kBN - 1) / kBN);
   if (tiles >= (int64_t)1 << 31) return cudaErrorInvalidValue;
   int64_t clusters = (sms < kMaxCtas ? sms : kMaxCtas) / 2;
-  {
-    // persistent grid: no more clusters than can be resident at once
-    static int resident[3][3] = {};
-    if (resident[kMode][ti] == 0) {
-      cudaLaunchConfig_t cfg = {};
-      cfg.gridDim = dim3((unsigned)(2 * clusters));
-      cfg.blockDim = dim3(kThreads);
-      cfg.dynamicSmemBytes = kSmemBytes;
-      cudaLaunchAttribute at[1];
-      at[0].id = cudaLaunchAttributeClusterDimension;
-      at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-      cfg.attrs = at; cfg.numAttrs = 1;
-      int n = 0;
-      if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n < 1) { (void)cudaGetLastError(); n = (int)clusters; }
-      resident[kMode][ti] = n;
-    }
-    if (resident[kMode][ti] < clusters) clusters = resident[kMode][ti];
+  if (cap == 0) {
+    if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes)) != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * clusters));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n < 1) { (void)cudaGetLastError(); n = (int)clusters; }
+    cap = n;
+    if (dev < kMaxDevices) resident[dev].store(cap, std::memory_order_release);
   }
+  if (cap < clusters) clusters = cap;
   if (tiles < clusters) clusters = tiles;
   return launch_pdl(kern, (unsigned)(2 * clusters), kThreads, kSmemBytes, s, map, a, (int)(box_m * kBK));
 }
 
 }  // namespace
 
-cudaError_t launch_gemm_tc2(const GemmArgs& a, cudaStream_t s) {
+bool gemm_tc_supported(int64_t M, int64_t K, int64_t N, int G) {
+  return M >= 1 && N >= 1 && G >= 1 && K % kBK == 0 && (K / G) % kBK == 0 && K / kBK < (1 << 24);
+}
+
+// Per-CTA fp32 running sums of the grouped epilogue: two CTAs per 256 x 256 tile.
+size_t gemm_tc_scratch_bytes(int64_t M, int64_t N, int G) {
+  if (G <= 1 || M <= 0 || N <= 0) return 0;
+  int64_t ctas = 2 * ((M + kPairM - 1) / kPairM) * ((N + kBN - 1) / kBN);
+  if (ctas > kMaxCtas) ctas = kMaxCtas;
+  return (size_t)ctas * kScratchPerCta;
+}
+
+cudaError_t launch_gemm_tc(const GemmArgs& a, cudaStream_t s) {
   if (a.y == nullptr) return launch<0, float>(a, s);
   const bool ext = a.beta_rows > 0 || a.relu || a.residual != nullptr || (a.ld_y > 0 && a.ld_y != a.N);
   switch (a.yt) {

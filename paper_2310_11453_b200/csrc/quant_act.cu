@@ -11,6 +11,7 @@
 // Per-tensor scope splits in two kernels: the first leaves each segment's moments in the
 // workspace and folds the extremes of x^ into a global atomic min/max on an order-preserving
 // encoding (order-independent, hence deterministic); the second re-reads x and writes codes.
+#include <algorithm>
 #include <atomic>
 #include <mutex>
 #include <random>
@@ -472,8 +473,8 @@ template <typename T>
 __global__ void __launch_bounds__(kRowWarps * 32, 1)
 rows_tensor_fused(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg, int mode, float ln_eps,
                   double inv_kg, ScopePartial* __restrict__ partials, SegRecord* __restrict__ recs,
-                  unsigned long long* __restrict__ tags, unsigned long long tag, uint32_t* __restrict__ status,
-                  int clear_status, int8_t* __restrict__ x_q, float* __restrict__ gamma, float* __restrict__ eta) {
+                  unsigned long long* __restrict__ tags, unsigned long long tag, unsigned long long wait_tag,
+                  unsigned meet_polls, uint32_t* __restrict__ status, int clear_status, int8_t* __restrict__ x_q, float* __restrict__ gamma, float* __restrict__ eta) {
   extern __shared__ __align__(16) unsigned char stage[];
   __shared__ int counter1, counter2;
   __shared__ unsigned long long part_lo[BL_MAX_GROUPS], part_hi[BL_MAX_GROUPS];
@@ -552,8 +553,8 @@ rows_tensor_fused(const T* __restrict__ x, int64_t segments, int64_t K, int G, i
   if (threadIdx.x < gridDim.x) {
     here = false;
     unsigned long long t0 = 0;
-    for (unsigned it = 0; it < kMeetSpins; ++it) {
-      if (ld_acquire_u64(tags + threadIdx.x) == tag) { here = true; break; }
+    for (unsigned it = 0; it <= meet_polls; ++it) {
+      if (ld_acquire_u64(tags + threadIdx.x) == wait_tag) { here = true; break; }
       if ((it & 63u) == 63u) {
         unsigned long long now;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
@@ -669,15 +670,20 @@ cudaError_t launch_fused(const QuantArgs& a, cudaStream_t s, const T* x, int64_t
   static std::atomic<int> with_pdl{1};                          // dropped for good if the pair is refused once
   cfg.numAttrs = with_pdl.load() ? 2 : 1;
   const unsigned long long tag = next_tag();
+  // test hook: a smaller poll limit, and a tag to wait for that no CTA publishes (the complement of this
+  // call's tag: the array holds this call's tag or those of earlier calls, whose high half is the same)
+  const long long dbg_polls = g_debug_wait_polls.load(std::memory_order_relaxed);
+  const unsigned meet_polls = dbg_polls < 0 ? kMeetSpins : (unsigned)std::min<long long>(dbg_polls, kMeetSpins);
+  const unsigned long long wait_tag = g_debug_meet_skew.load(std::memory_order_relaxed) ? ~tag : tag;
   const int clear = a.keep_status ? 0 : 1;
   e = cudaLaunchKernelEx(&cfg, kern, x, segments, a.K, a.G, Kg, (int)a.mode, a.ln_eps, inv_kg, partials, recs, tags,
-                         tag, status, clear, a.x_q, a.gamma, a.eta);
+                         tag, wait_tag, meet_polls, status, clear, a.x_q, a.gamma, a.eta);
   if (e != cudaSuccess && cfg.numAttrs == 2) {
     (void)cudaGetLastError();
     with_pdl.store(0);
     cfg.numAttrs = 1;
     e = cudaLaunchKernelEx(&cfg, kern, x, segments, a.K, a.G, Kg, (int)a.mode, a.ln_eps, inv_kg, partials, recs, tags,
-                           tag, status, clear, a.x_q, a.gamma, a.eta);
+                           tag, wait_tag, meet_polls, status, clear, a.x_q, a.gamma, a.eta);
   }
   return e;
 }

@@ -30,6 +30,7 @@ def test_gemv_decode_batch(M, K, N, G, dtype, mode, relu):
     omode = O.ETA if mode == "eta" else O.ABSMAX
     w_ref = O.binarize(W.numpy(), G=G)
     w_gpu = B.binarize_pack(W.to(DEV), G=G, layout=B.DECODE)
+    torch.cuda.synchronize()
     xd = x.to(DEV)
     # The kernel quantises the tokens itself and its codes cannot be read back, so the comparison
     # allows what the quantising kernels are allowed: a different neighbour at a rounding tie,
@@ -81,6 +82,7 @@ def test_gemv_decode_batch_integer_definition_exactly():
     W = synth.make_w(N, K, torch.float32, seed=9)
     w_ref = O.binarize(W.numpy())
     w_gpu = B.binarize_pack(W.to(DEV), layout=B.DECODE)
+    torch.cuda.synchronize()
     y = B.gemv_decode_batch(x.to(DEV), w_gpu["W_packed"], w_gpu["beta"], N, ln_eps=-1.0, out_dtype=torch.float32)
     c = codes.numpy().copy()
     c[:, 0] = 127

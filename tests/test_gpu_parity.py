@@ -400,7 +400,48 @@ def test_forward_eta_correction():
                          eta_correction=True)
 
 
+def test_bounded_wait_that_runs_out_is_reported_and_the_next_call_recovers():
+    # The cooperative per-tensor kernel's CTAs meet between its two passes with a bounded wait.  The
+    # test hook makes them wait (a few hundred polls) for an arrival tag that nobody publishes: the
+    # wait must run out, the kernel must return with BL_ERR_TIMEOUT in the status word and without
+    # writing codes, and the next ordinary call on the same workspace must be clean again.
+    M, K = 1024, 2048
+    x = synth.make_x(M, K, torch.bfloat16, seed=77, outliers=True).to(DEV)
+    ws = torch.zeros(B.workspace_bytes(B.OP_QUANT_ACT, M, 1, K, 1), dtype=torch.uint8, device=DEV)
+    good = B.quant_act(x, gran=B.PER_TENSOR, ln_eps=1e-5, ws=ws)
+    assert B.ws_status(ws) == B.OK
+    want = good["x_q"].clone()
+    out = dict(x_q=torch.full((M, K), 99, dtype=torch.int8, device=DEV),
+               gamma=torch.zeros(1, device=DEV), eta=torch.zeros(1, device=DEV))
+    try:
+        B.debug_wait_limit(300, meet_skew=True)
+        B.quant_act(x, gran=B.PER_TENSOR, ln_eps=1e-5, out=out, ws=ws)
+        status = B.ws_status(ws)                       # synchronises: the kernel has returned
+    finally:
+        B.debug_wait_limit(-1)
+    assert status == B.ERR_TIMEOUT
+    assert bool((out["x_q"] == 99).all()), "codes were written although the meeting failed"
+    again = B.quant_act(x, gran=B.PER_TENSOR, ln_eps=1e-5, out=out, ws=ws)
+    assert B.ws_status(ws) == B.OK
+    assert torch.equal(again["x_q"], want)
+
+
 # ---------------------------------------------------------------- decode GEMV
+
+def explained_by_code_flips(err, signs, step, tol, max_flips):
+    """True when the output error of one token is, up to `tol`, a sum of at most `max_flips` single
+    code changes of +-1: changing code k by one moves output n by W~[n,k] * step[k].  err [N];
+    signs [N,K] in {-1,+1}; step [K] (the quantisation step of feature k's group).  The kernel
+    quantises x itself, so its codes cannot be read back; they can be inferred this way."""
+    r = np.array(err, np.float64)
+    for _ in range(max_flips + 1):
+        if np.abs(r).max() <= tol:
+            return True
+        score = (signs * r[:, None]).sum(axis=0) / (signs.shape[0] * step)       # about +-1 at a flipped code
+        k = int(np.abs(score).argmax())
+        r = r - np.sign(score[k]) * step[k] * signs[:, k]
+    return False
+
 
 @pytest.mark.parametrize("K,N,G,dtype,mode,relu", [
     (4096, 16384, 1, "f16", "absmax", False),      # config c2
@@ -409,6 +450,12 @@ def test_forward_eta_correction():
     (8192, 2048, 1, "bf16", "absmax", False),      # two K slices per row
     (28672, 112, 8, "bf16", "eta", True),          # c5-shaped K, seven slices
     (2560, 80, 1, "f16", "absmax", False),         # K not a multiple of the slice
+    (1024, 40960, 1, "f16", "absmax", False),      # more weight stages than the shared-memory ring holds
+    (512, 49152, 2, "bf16", "eta", True),          # the same with groups and row terms
+    (32768, 32, 1, "f16", "absmax", False),        # the longest row: one row slot, eight slices
+    (4096, 16384, 1, "bf16", "eta", True),         # c2-shaped, eta form (with and without the row terms)
+    (12288, 4096, 1, "f16", "absmax", False),      # three slices per row
+    (4096, 160000, 1, "f16", "absmax", False),     # 1082 rows per CTA: the ring is refilled many times
 ])
 def test_gemv_decode(K, N, G, dtype, mode, relu):
     x = synth.make_x(1, K, DT[dtype], seed=K + N, outliers=False, relu=relu)
@@ -416,27 +463,27 @@ def test_gemv_decode(K, N, G, dtype, mode, relu):
     omode = O.ETA if mode == "eta" else O.ABSMAX
     w_ref = O.binarize(W.numpy(), G=G)
     w_gpu = B.binarize_pack(W.to(DEV), G=G, layout=B.DECODE)
+    torch.cuda.synchronize()                       # the decode kernel reads the weights ahead of stream order
+    signs = None
     for corr in ([False, True] if mode == "eta" else [False]):
         y = B.gemv_decode(x.to(DEV), w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode, ln_eps=1e-5,
                           rowsum=w_gpu["rowsum"], eta_correction=corr, out_dtype=torch.float32)
         ref = O.forward(as_f32_np(x), w_ref["bits"], w_ref["beta"], G=G, mode=omode, gran=O.PER_TOKEN,
                         ln_eps=1e-5, rowsum=w_ref["rowsum"], eta_correction=corr)
-        q = B.quant_act(x.to(DEV), G=G, mode=omode, gran=B.PER_TOKEN, ln_eps=1e-5)
         torch.cuda.synchronize()
-        diff = check_codes(q["x_q"].cpu().numpy(), ref["codes"], x=as_f32_np(x), G=G,
-                           eta_per_token=(mode == "eta"))
         rms = np.sqrt((ref["y"] ** 2).mean())
-        step = (w_ref["beta"] * ref["gamma"][0] / 128.0).max()
-        # the kernel quantises x itself; allow one step per code that may have flipped (same
-        # allowance as the quant kernel: at most 1e-4 of K, at least one)
+        err = y.cpu().numpy().astype(np.float64) - ref["y"][0]
+        if np.abs(err).max() <= FLOAT_TOL_RMS * rms:
+            continue
+        # Not within the plain tolerance: the only accepted reason is that a few codes of the token
+        # sit one step away from the oracle's (at most 1e-4 of K, at least one; exact ties of the
+        # eta form, where either neighbour is right, on top).  No slack is granted otherwise.
+        if signs is None:
+            signs = 2.0 * np.unpackbits(w_ref["bits"], axis=1, bitorder="little")[:, :K].astype(np.float64) - 1.0
+        step = np.repeat(w_ref["beta"] * ref["gamma"][0] / 128.0, K // G)
         ties = count_exact_ties(as_f32_np(x)[0], G) if mode == "eta" else 0
-        slack = (max(1, int(CODE_FLIP_FRACTION * K)) + ties) * step
-        y_gpu = y.cpu().numpy().astype(np.float64)
-        assert np.abs(y_gpu - ref["y"][0]).max() <= FLOAT_TOL_RMS * rms + slack
-        # typical error is far below the bound: the median element must meet the plain tolerance
-        # (an exact tie that went the other way moves every output of the token by one step)
-        if ties == 0:
-            assert np.median(np.abs(y_gpu - ref["y"][0])) <= FLOAT_TOL_RMS * rms
+        assert explained_by_code_flips(err, signs, step, FLOAT_TOL_RMS * rms, max(1, int(CODE_FLIP_FRACTION * K)) + ties), \
+            f"decode output differs from the oracle by {np.abs(err).max():.3e} (rms {rms:.3e}) and no few code flips explain it"
     y16 = B.gemv_decode(x.to(DEV), w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode, ln_eps=1e-5,
                         out_dtype=DT[dtype])
     y32 = B.gemv_decode(x.to(DEV), w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode, ln_eps=1e-5,
@@ -444,10 +491,28 @@ def test_gemv_decode(K, N, G, dtype, mode, relu):
     assert torch.equal(y16, y32.to(DT[dtype]))
 
 
-def test_gemv_decode_matches_integer_definition_exactly():
+def test_gemv_decode_weights_from_global_memory_when_the_wait_runs_out():
+    # With the poll limit of the kernel's one bounded wait at zero, warps whose weight stage has not
+    # landed at their first look read it from global memory instead: same bits, same y.
+    for K, N in [(4096, 16384), (1024, 40960), (8192, 2048)]:
+        x = synth.make_x(1, K, torch.float16, seed=K, outliers=False).to(DEV)
+        w = B.binarize_pack(synth.make_w(N, K, torch.float32, seed=K + 1).to(DEV), layout=B.DECODE)
+        torch.cuda.synchronize()
+        want = B.gemv_decode(x, w["W_packed"], w["beta"], N, out_dtype=torch.float32)
+        try:
+            B.debug_wait_limit(0)
+            got = [B.gemv_decode(x, w["W_packed"], w["beta"], N, out_dtype=torch.float32) for _ in range(3)]
+        finally:
+            B.debug_wait_limit(-1)
+        torch.cuda.synchronize()
+        for g in got:
+            assert torch.equal(g, want)
+
+
+@pytest.mark.parametrize("K,N", [(1024, 64), (4096, 160), (8192, 48)])
+def test_gemv_decode_matches_integer_definition_exactly(K, N):
     # With LN skipped and gamma planted at 128 the codes are the inputs themselves, so the
     # output must equal acc * beta exactly as computed by the oracle's integer matmul.
-    K, N = 1024, 64
     codes = synth.make_codes(1, K, seed=5)
     codes[0, 0] = 127
     x = codes.float()
@@ -455,6 +520,7 @@ def test_gemv_decode_matches_integer_definition_exactly():
     W = synth.make_w(N, K, torch.float32, seed=6)
     w_ref = O.binarize(W.numpy())
     w_gpu = B.binarize_pack(W.to(DEV), layout=B.DECODE)
+    torch.cuda.synchronize()
     y = B.gemv_decode(x.to(DEV), w_gpu["W_packed"], w_gpu["beta"], N, ln_eps=-1.0, out_dtype=torch.float32)
     c = codes.clone()
     c[0, 1] = 127
