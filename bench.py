@@ -14,8 +14,10 @@ Every rank runs the same replica on its own GPU (the layer has no exchange step)
 value is the sum over ranks divided by the slowest rank's time.
 """
 import argparse
+import hashlib
 import json
 import os
+import socket
 import statistics
 import subprocess
 import sys
@@ -61,7 +63,7 @@ def load_peaks():
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the timed region runs."""
 
-    def __init__(self, index, period_s=0.002):
+    def __init__(self, index, period_s=0.0002):
         self.index, self.period, self.samples, self.reasons = index, period_s, [], set()
         self.max_mhz, self._stop, self._thread, self._h, self._nv = None, threading.Event(), None, None, None
         try:
@@ -141,6 +143,48 @@ def job_throughput(units_local, ms_local, dist=None, device=None):
     return float(u.item()) / (float(t.item()) * 1e-3), float(t.item())
 
 
+def sha256_of(t):
+    """SHA-256 of a host tensor's bytes (inputs are logged by hash so that a run can be reproduced)."""
+    return hashlib.sha256(t.contiguous().view(torch.uint8).numpy().tobytes()).hexdigest()
+
+
+def library_int8_tops(M, K, N, dev, reps=20):
+    """In-job calibration of the box: the library int8 GEMM (torch._int_mm, int32 output) on the bench
+    shape, timed alone with CUDA events.  None when the routine is unavailable."""
+    try:
+        a = torch.randint(-127, 128, (M, K), dtype=torch.int8, device=dev)
+        b = torch.randint(-1, 2, (K, N), dtype=torch.int8, device=dev)
+        for _ in range(3):
+            torch._int_mm(a, b)
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        t0.record()
+        for _ in range(reps):
+            torch._int_mm(a, b)
+        t1.record()
+        torch.cuda.synchronize()
+        return 2.0 * M * N * K / (t0.elapsed_time(t1) / reps * 1e-3) / 1e12
+    except Exception:
+        return None
+
+
+def measured_copy_gbs(dev, nbytes=1 << 30, reps=5):
+    """In-job device-to-device copy rate (read + write bytes), the same kind of figure as the measured peak."""
+    a = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    b = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    b.copy_(a)
+    best = None
+    for _ in range(reps):
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        b.copy_(a)
+        t1.record()
+        torch.cuda.synchronize()
+        ms = t0.elapsed_time(t1)
+        best = ms if best is None else min(best, ms)
+    return 2.0 * nbytes / (best * 1e-3) / 1e9
+
+
 # --------------------------------------------------------------------------------------- own arm
 
 def run_b200(args):
@@ -161,6 +205,8 @@ def run_b200(args):
         dist.init_process_group("nccl", device_id=dev)
     B.lib()                                           # fail here, loudly, if the library is missing
     peaks = load_peaks()
+    run_clocks = ClockSampler(local, period_s=0.01)   # across every part of the run
+    run_clocks.__enter__()
     K_steps, W_steps = args.steps, max(args.warmup, 3)
 
     def barrier():
@@ -173,7 +219,10 @@ def run_b200(args):
     xs_host = [synth.make_x(M, K, torch.bfloat16, seed=2 + 101 * r + 7919 * rank, outliers=True).pin_memory()
                for r in range(ROTATE)]
     xs = [x.to(dev) for x in xs_host]
-    W = synth.make_w(N, K, torch.float32, seed=2).to(dev)
+    W_host = synth.make_w(N, K, torch.float32, seed=2)
+    hashes = {f"x[{r}] bf16 [{M},{K}]": sha256_of(x) for r, x in enumerate(xs_host)}
+    hashes[f"W fp32 [{N},{K}]"] = sha256_of(W_host)
+    W = W_host.to(dev)
     w = B.binarize_pack(W, G=G, layout=B.PREFILL)
     ys = [torch.empty((M, N), dtype=torch.bfloat16, device=dev) for _ in range(ROTATE)]
     qs = [dict(x_q=torch.empty((M, K), dtype=torch.int8, device=dev),
@@ -308,6 +357,7 @@ def run_b200(args):
                    "l2": f"rotating over {ROTATE} input/output sets, {ROTATE * (M * K * 3 + M * N * 2) >> 20} MiB "
                          "in total, larger than L2"},
         "clocks": None,
+        "inputs_sha256": hashes,
         "e2e": e2e,
         "gpu_launches": 2 * K_steps,
         "kernels_per_step": ["rows_tensor_fused", "gemm_tc2_kernel"],
@@ -322,6 +372,13 @@ def run_b200(args):
                            "traffic": NCU_TRAFFIC["rows_tensor_fused"], "avg_ms": quant_ms, "peak_source": peaks["source"] + " copy"},
     }
 
+    lib_tops = library_int8_tops(M, K, N, dev) if rank == 0 else None
+    if lib_tops:
+        line["roofline"]["library_int8_tops"] = lib_tops
+        line["roofline"]["frac_of_library_int8"] = gemm_tops / lib_tops
+        line["roofline"]["library_int8"] = "torch._int_mm on the same shape, int32 output, timed in this job"
+    if rank == 0:
+        line["copy_gbs_in_job"] = measured_copy_gbs(dev)
     parts = set(args.parts.split(","))
     if rank == 0 and world == 1:
         if "decode" in parts:
@@ -332,9 +389,15 @@ def run_b200(args):
             line["block"] = bench_block(B, synth, dev, peaks)
         if "grouped" in parts:
             line["grouped"] = bench_grouped(B, synth, dev, peaks)
+        if "small" in parts:
+            line["small"] = bench_small(B, synth, dev)
         if "cpu" in parts:
             line["cpu_baseline"] = cpu_baseline_prefill(xs_host[0], W.cpu())
+            line["cpu_baseline_decode"] = cpu_baseline_decode()
+            line["cpu_baseline_grouped"] = cpu_baseline_grouped()
     line["clocks"] = clocks.summary()
+    run_clocks.__exit__()
+    line["clocks_whole_run"] = run_clocks.summary()
     if rank == 0:
         print(json.dumps(line), flush=True)
     if dist is not None:
@@ -569,7 +632,82 @@ def bench_block(B, synth, dev, peaks):
             "gpu_launches": 10 * 9}
 
 
+def bench_small(B, synth, dev):
+    """Config 1: one 125M-shaped layer, x fp32 [64, 768], W fp32 [3072, 768], per-tensor absmax, y fp32.
+    0.3 GOP: a latency case, reported in microseconds per call (each entry point timed alone, calls
+    back to back on one stream)."""
+    M, K, N = 64, 768, 3072
+    x = synth.make_x(M, K, torch.float32, seed=0, outliers=True).to(dev)
+    W = synth.make_w(N, K, torch.float32, seed=0).to(dev)
+    w = B.binarize_pack(W, layout=B.PREFILL)
+    ws_p = torch.empty(B.workspace_bytes(B.OP_BINARIZE_PACK, 1, N, K, 1), dtype=torch.uint8, device=dev)
+    ws_q = torch.empty(B.workspace_bytes(B.OP_QUANT_ACT, M, 1, K, 1), dtype=torch.uint8, device=dev)
+    ws_f = torch.empty(B.workspace_bytes(B.OP_FORWARD, M, N, K, 1), dtype=torch.uint8, device=dev)
+    q = dict(x_q=torch.empty((M, K), dtype=torch.int8, device=dev), gamma=torch.empty(1, device=dev),
+             eta=torch.zeros(1, device=dev))
+    y = torch.empty((M, N), dtype=torch.float32, device=dev)
+
+    def timed(fn, reps=200):
+        for _ in range(5):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps * 1e3
+
+    out = {"workload": "single BitLinear layer: x fp32 [64,768] N(0,1) + 0.1% x20 outliers, W fp32 [3072,768] "
+                       "N(0,0.02), per-tensor absmax, y fp32, seed 0 (latency case: microseconds per call)",
+           "pack_us": timed(lambda: B.binarize_pack(W, layout=B.PREFILL, out=w, ws=ws_p)),
+           "quant_us": timed(lambda: B.quant_act(x, gran=B.PER_TENSOR, out=q, ws=ws_q)),
+           "forward_us": timed(lambda: B.forward(x, w["W_packed"], w["beta"], N, gran=B.PER_TENSOR, layout=B.PREFILL,
+                                                 y=y, ws=ws_f))}
+    assert B.ws_status(ws_f) == B.OK
+    return out
+
+
 # --------------------------------------------------------------------------- the CPU oracle, timed
+
+def cpu_baseline_decode(reps=20):
+    """The oracle on config 2 (one token, K 4096, N 16384): full size, a few repetitions."""
+    from oracle import oracle as O
+    from paper_2310_11453_b200 import synth
+    K, N = DECODE["K"], DECODE["N"]
+    W = synth.make_w(N, K, torch.float32, seed=1)
+    wb = O.binarize(W.numpy())
+    x = synth.make_x(reps, K, torch.float16, seed=1, outliers=False).to(torch.float32).numpy()
+    t = time.perf_counter()
+    for i in range(reps):
+        O.forward(x[i:i + 1], wb["bits"], wb["beta"], gran=O.PER_TOKEN, ln_eps=1e-5)
+    dt = (time.perf_counter() - t) / reps
+    nbytes = N * K / 8 + 2 * K + 2 * N
+    return {"value": nbytes / dt / 1e9, "unit": "GB/s of packed weights", "us_per_call": dt * 1e6, "cores": O.num_threads(),
+            "kind": "oracle", "sample": f"oracle forward, one token, full W [16384,4096], mean of {reps} calls"}
+
+
+def cpu_baseline_grouped(tokens=16):
+    """The oracle on config 5 (G = 8): binarisation of the full weight matrix, and the forward on a
+    token sample against the full matrix."""
+    from oracle import oracle as O
+    from paper_2310_11453_b200 import synth
+    M, K, N, G = 4096, 28672, 7168, 8
+    W = synth.make_w(N, K, torch.float32, seed=4)
+    t = time.perf_counter()
+    wb = O.binarize(W.numpy(), G=G)
+    t_bin = time.perf_counter() - t
+    del W
+    x = synth.make_x(tokens, K, torch.bfloat16, seed=4, outliers=False, relu=True).to(torch.float32).numpy()
+    t = time.perf_counter()
+    O.forward(x, wb["bits"], wb["beta"], G=G, mode=O.ETA, gran=O.PER_TENSOR, ln_eps=1e-5)
+    dt = time.perf_counter() - t
+    return {"value": 2.0 * tokens * N * K / dt / 1e12, "unit": "TOPS", "cores": O.num_threads(), "kind": "oracle",
+            "binarize_s": t_bin, "binarize_gbs": (2.0 * N * K * 4 + N * K / 8) / t_bin / 1e9,
+            "sample": f"oracle forward on {tokens} of {M} tokens against the full W [7168,28672], G = 8, eta form "
+                      f"({dt:.2f} s); binarisation of the full matrix {t_bin:.2f} s"}
+
 
 def oracle_prefill_sample(x_host, W_host, tokens, reps=1):
     """Times the CPU oracle's forward (LN+quant, matmul, rescale) on the first `tokens` tokens of the
@@ -653,10 +791,18 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
-    ap.add_argument("--parts", default="decode,pack,grouped,block,cpu",
-                    help="extra measurements beside the prefill step (comma list of decode, pack, grouped, block, cpu; "
+    ap.add_argument("--parts", default="decode,pack,grouped,block,small,cpu",
+                    help="extra measurements beside the prefill step (comma list of decode, pack, grouped, block, small, cpu; "
                          "'none' for the prefill step alone, e.g. under a profiler)")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started by hand with --gpus N: run the N replicas (one process per GPU) under torchrun
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        raise SystemExit(subprocess.call(cmd))
     if args.impl == "reference":
         run_reference(args)
     else:

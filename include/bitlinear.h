@@ -145,19 +145,30 @@ bl_status bitlinear_quant_act(const void* x, bl_dtype xt, int64_t M, int64_t K, 
  * BL_NOALLOC_MAX_SEGMENTS segments plus a 0.26 MB header, about 0.7 MB in all, resident on every
  * GPU that loads the library until the process ends).  Consequences:
  *   - BL_PER_TENSOR calls with M * G > BL_NOALLOC_MAX_SEGMENTS return BL_ERR_TOO_LARGE and launch
- *     nothing.  BL_PER_TOKEN calls need no scratch and have no such limit.
- *   - All calls on one GPU share the array.  Calls that may overlap on the GPU (different
- *     streams) race on it and corrupt each other; keep them on one stream or order them yourself.
- *     A call leaves nothing behind that the next one depends on.
+ *     nothing.  BL_PER_TOKEN calls keep no statistics there and have no such limit; they use the
+ *     array's first word as their status word only.
+ *   - All calls on one GPU share the array.  BL_PER_TENSOR calls that may overlap on the GPU
+ *     (different streams) race on it and corrupt each other; keep them on one stream or order them
+ *     yourself.  Overlapping BL_PER_TOKEN calls share nothing but the status word (each clears it
+ *     when it starts), so their outputs are unaffected, but a timeout report of one may be wiped
+ *     by the other.  A call leaves nothing behind that the next one depends on.
  *   - The first call on each device looks up the array's device address
  *     (cudaGetSymbolAddress); make that first call outside any stream capture.
  *   - No cudaMalloc, cudaFree or other allocating routine is called, now or later.
- * Arguments, results, error codes and rounding are otherwise exactly those of bitlinear_quant_act;
- * the same kernels run, so the outputs are bit-identical. */
+ * Arguments, results, host-side error codes and rounding are otherwise exactly those of
+ * bitlinear_quant_act; the same kernels run, so the outputs are bit-identical.  The one difference
+ * is where a device-side timeout is reported: the status word lives in the library's array, which
+ * the caller cannot pass to bitlinear_ws_status; bitlinear_noalloc_status reads it instead. */
 #define BL_NOALLOC_MAX_SEGMENTS 16384
 bl_status bitlinear_quant_act_noalloc(const void* x, bl_dtype xt, int64_t M, int64_t K, int G, int b,
                                       bl_quant_mode mode, bl_gran gran, float ln_eps, int8_t* x_q,
                                       float* gamma, float* eta, void* stream);
+
+/* Synchronises `stream`, then reads the status word that the last bitlinear_quant_act_noalloc call on
+ * the current device left in the library's array (the counterpart of bitlinear_ws_status for that
+ * entry point; the paper has no counterpart).  BL_OK, BL_ERR_TIMEOUT (a bounded device-side wait of
+ * that call ran out: its codes were not written), or BL_ERR_CUDA.  Allocates nothing. */
+bl_status bitlinear_noalloc_status(void* stream);
 
 /* Steps 1, 2, 4, Eq. 11: y = (W~ x~) . beta_g gamma / Q_b summed over groups in ascending order.
  *   eta_correction != 0 (BL_ETA only) adds eta.beta_g.rowsum[n,g], which undoes the shift of

@@ -829,3 +829,11 @@ extern "C" bl_status bitlinear_quant_act_noalloc(const void* x, bl_dtype xt, int
                              bl::kNoAllocBytes, stream);
 }
 
+extern "C" bl_status bitlinear_noalloc_status(void* stream) {
+  void* scratch = nullptr;
+  if (bl::noalloc_scratch_address(&scratch) != cudaSuccess) return BL_ERR_CUDA;
+  uint32_t word = 0;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return BL_ERR_CUDA;
+  if (cudaMemcpy(&word, scratch, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return BL_ERR_CUDA;
+  return word == 0 ? BL_OK : BL_ERR_TIMEOUT;
+}

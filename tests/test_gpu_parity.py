@@ -53,14 +53,23 @@ def self_scaled_rows(x, G, ln_eps=1e-5):
     return out
 
 
+TIE_EXEMPT_FRACTION = 1e-2      # cap on the elements that may be excused as exact ties
+TIE_LOG = []                     # (elements, differing, excused as exact ties, of those at the even neighbour)
+
+
 def check_codes(gpu_codes, ref_codes, x=None, G=1, eta_per_token=False, eta_per_tensor=False):
     """+-1 on at most 1e-4 of the elements.  Elements whose exact value is a mathematical tie
     (decidable where LN cancels and the value is rational: the per-token eta form, and in the
     per-tensor eta form the segment that holds both extremes of its scope) are valid either way
-    and are not counted."""
+    and are not counted against that bar; their number is capped (1e-2 of the elements, at least
+    4), recorded in TIE_LOG and printed, together with how many of them the GPU sent to the even
+    neighbour (what round-half-to-even does when the tie survives the arithmetic).  Such ties are
+    not rare with 16-bit inputs: when the segment's range max - min has few mantissa bits, every
+    input whose last mantissa bit falls right is one (0.3 % of the elements in one case of the
+    seeded sweep, half of which the kernel sent to the even neighbour: LN's rounding noise decides)."""
     diff = gpu_codes.astype(np.int32) - ref_codes.astype(np.int32)
     assert np.abs(diff).max() <= 1, "a code differs by more than one step"
-    counted = 0
+    counted = excused = to_even = 0
     rows = self_scaled_rows(x, G) if (eta_per_tensor and x is not None and np.count_nonzero(diff)) else set()
     for m, k in zip(*np.nonzero(diff)):
         if x is not None and (eta_per_token or rows):
@@ -68,8 +77,16 @@ def check_codes(gpu_codes, ref_codes, x=None, G=1, eta_per_token=False, eta_per_
             g = k // Kg
             if (eta_per_token or (int(m), int(g)) in rows) and \
                     exact_tie_per_token_eta(x[m, g * Kg:(g + 1) * Kg], k - g * Kg):
+                excused += 1
+                to_even += int(gpu_codes[m, k]) % 2 == 0
                 continue
         counted += 1
+    TIE_LOG.append((diff.size, int(np.count_nonzero(diff)), excused, to_even))
+    if excused:
+        print(f"check_codes: {excused} of {diff.size} elements excused as exact ties "
+              f"({to_even} at the even neighbour), {counted} counted")
+    assert excused <= max(4, int(TIE_EXEMPT_FRACTION * diff.size)), \
+        f"{excused} of {diff.size} code differences claimed as exact ties"
     assert counted <= max(1, int(CODE_FLIP_FRACTION * diff.size)), f"{counted} of {diff.size} codes differ"
     return diff
 
@@ -256,18 +273,15 @@ _HAVE_TC = None
 
 
 def have_tensor_core_path():
-    """True once the PREFILL (tcgen05) kernel is compiled in; probed with a valid tiny call."""
+    """The PREFILL (tcgen05) kernel is always compiled in: a valid tiny call must succeed, so that the
+    bit-exact GEMM and forward tests can never go green on the CUDA-core kernel alone."""
     global _HAVE_TC
     if _HAVE_TC is None:
         xq = torch.zeros((128, 128), dtype=torch.int8, device=DEV)
         wp = torch.zeros(B.packed_bytes(B.PREFILL, 128, 128), dtype=torch.uint8, device=DEV)
-        try:
-            B.matmul_i32(xq, wp, 128, layout=B.PREFILL)
-            _HAVE_TC = True
-        except B.BitLinearError as e:
-            assert e.code == 2
-            _HAVE_TC = False
+        B.matmul_i32(xq, wp, 128, layout=B.PREFILL)         # raises if the tensor-core path refuses a valid shape
         torch.cuda.synchronize()
+        _HAVE_TC = True
     return _HAVE_TC
 
 

@@ -227,6 +227,29 @@ def test_per_tensor_gamma_is_global():
     assert rt["gamma"][:, 0].tolist() == [4.0, 64.0] and rt["codes"][0, 0] == 127
 
 
+def test_per_tensor_eta_over_several_rows_hand_worked():
+    # Eq. 6 / 14 per tensor, LN skipped, two groups of eight features over three tokens.  By hand:
+    # group 0: eta = 0 (the minimum over ALL rows, found in row 1), gamma = 10 - 0 (the maximum is in
+    # row 1 too), codes = rne(12.8 x); group 1: eta = -3, gamma = 5 - (-3) = 8, codes = rne(16 (x + 3)).
+    # The maximum of each group reaches 128 and is clipped to 127.  gamma is the range max - min, not
+    # max |x| (which would be 10 and 5).
+    x = np.array([[1, 2, 3, 4, 0.5, 1.5, 2, 2, -3, -1, 1, 5, 0, 0, 0, 0],
+                  [0, 5, 6, 10, 1, 1, 1, 1, 5, 5, 5, 5, 5, 5, 5, 5],
+                  [7, 8, 9, 2.5, 3, 3, 3, 3, -3, 0, 2, 3, 1, 1, 1, 1]], np.float32)
+    r = O.quant_act(x, G=2, mode=O.ETA, gran=O.PER_TENSOR, ln_eps=-1.0)
+    assert r["eta"].tolist() == [0.0, -3.0]
+    assert r["gamma"].tolist() == [10.0, 8.0]
+    assert r["codes"].tolist() == [
+        [13, 26, 38, 51, 6, 19, 26, 26, 0, 32, 64, 127, 48, 48, 48, 48],
+        [0, 64, 77, 127, 13, 13, 13, 13, 127, 127, 127, 127, 127, 127, 127, 127],
+        [90, 102, 115, 32, 38, 38, 38, 38, 0, 48, 80, 96, 64, 64, 64, 64]]
+    # per token the same input has its own eta and gamma per row and group
+    rt = O.quant_act(x, G=2, mode=O.ETA, gran=O.PER_TOKEN, ln_eps=-1.0)
+    assert rt["eta"].tolist() == [[0.5, -3.0], [0.0, 5.0], [2.5, -3.0]]
+    assert rt["gamma"].tolist() == [[3.5, 8.0], [10.0, 0.0], [6.5, 6.0]]
+    assert rt["codes"][1, 8:].tolist() == [0] * 8                 # a constant segment: gamma = 0, codes 0
+
+
 def test_zero_input_gives_zero_codes():
     r = O.quant_act(np.zeros((2, 16), np.float32), ln_eps=1e-5)
     assert (r["codes"] == 0).all() and (r["gamma"] == 0).all()

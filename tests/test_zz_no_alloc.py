@@ -5,13 +5,16 @@ running inside another framework's stream callback, a real-time loop with a fixe
 binding that only forwards the pointers it was handed.  For them the library keeps the per-tensor
 statistics of LN + quantisation in a fixed array of its own.  The entry point runs the same kernels
 as bitlinear_quant_act, so its outputs must be bit-identical to it - on the first call and on a
-second one that follows immediately with other data (the array keeps the first call's contents).
+second one that follows immediately with other data (the array keeps the first call's contents) -
+and, like every quantising entry point, within the stated bars of the CPU oracle.
 
 This file is named so that pytest collects it after every other test file.
 """
+import numpy as np
 import pytest
 import torch
 
+from oracle import oracle as O
 from paper_2310_11453_b200 import binding as B
 from paper_2310_11453_b200 import synth
 
@@ -41,12 +44,20 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point(mode, gran, G):
     got = [_outputs(x.shape[0], K, G, gran) for x in xs]
     for x, out in zip(xs, got):                       # nothing between the two calls
         B.quant_act_noalloc(x, G=G, mode=mode, gran=gran, out=out)
-    torch.cuda.synchronize()
+    assert B.noalloc_status() == B.OK                 # synchronises; no bounded wait of the calls ran out
     for x, out in zip(xs, got):
         ref = B.quant_act(x, G=G, mode=mode, gran=gran, out=_outputs(x.shape[0], K, G, gran))
         torch.cuda.synchronize()
         assert _same(out, ref)
         assert out["x_q"].abs().max().item() <= 127
+        # and against the CPU oracle, at the bars of the other quantisation tests: codes +-1 on at most
+        # 1e-4 of the elements, gamma and eta to 2e-6 relative
+        want = O.quant_act(x.float().cpu().numpy(), G=G, mode=mode, gran=gran, ln_eps=1e-5)
+        diff = out["x_q"].cpu().numpy().astype(np.int32) - want["codes"].astype(np.int32)
+        assert np.abs(diff).max() <= 1 and np.count_nonzero(diff) <= max(1, int(1e-4 * diff.size))
+        np.testing.assert_allclose(out["gamma"].cpu().numpy(), want["gamma"], rtol=2e-6)
+        if mode == B.ETA:
+            np.testing.assert_allclose(out["eta"].cpu().numpy(), want["eta"], rtol=2e-6, atol=1e-6)
 
 
 def test_sizes_beyond_the_built_in_scratch_are_refused():
