@@ -41,10 +41,11 @@ INT8_TO_BF16 = 2.0                                   # nominal dense int8 : bf16
 # profiles/, taken with ncu on these same workloads.  A figure is valid only while its kernel is the
 # one that was profiled: set it to None when the kernel changes, until the capture is redone.
 NCU_TRAFFIC = {
-    "gemm_tc2_kernel": 54.3e6,                       # 36.4 MB read + 17.9 MB written (y largely still in L2)
-    "rows_tensor_fused": 70.7e6,                     # 67.2 MB read + 3.5 MB written (second pass from smem and L2)
-    "gemv_decode_kernel": 8.45e6,
-    "reduce_partials + sign_pack": 135.8e6,          # 67.1 + 0.5 and 67.1 + 1.1 MB
+    "gemm_tc2_kernel": 54.2e6,                       # 36.5 MB read + 17.7 MB written (y largely still in L2)
+    "rows_tensor_fused": 70.3e6,                     # 67.2 MB read + 3.2 MB written (second pass from smem and L2)
+    "gemv_decode_fast_kernel": 8.43e6,
+    "reduce_partials + sign_pack_rows": 70.1e6,      # first pass 66.3 MB read, second pass served from L2
+                                                     # (capture without cache flushes between the launches)
 }
 
 
@@ -372,14 +373,14 @@ def run_b200(args):
                            "traffic": NCU_TRAFFIC["rows_tensor_fused"], "avg_ms": quant_ms, "peak_source": peaks["source"] + " copy"},
     }
 
-    lib_tops = library_int8_tops(M, K, N, dev) if rank == 0 else None
+    parts = set(args.parts.split(","))
+    lib_tops = library_int8_tops(M, K, N, dev) if rank == 0 and "calib" in parts else None
     if lib_tops:
         line["roofline"]["library_int8_tops"] = lib_tops
         line["roofline"]["frac_of_library_int8"] = gemm_tops / lib_tops
         line["roofline"]["library_int8"] = "torch._int_mm on the same shape, int32 output, timed in this job"
-    if rank == 0:
+    if rank == 0 and "calib" in parts:
         line["copy_gbs_in_job"] = measured_copy_gbs(dev)
-    parts = set(args.parts.split(","))
     if rank == 0 and world == 1:
         if "decode" in parts:
             line["decode"] = bench_decode(B, synth, dev, peaks)
@@ -513,8 +514,8 @@ def bench_decode(B, synth, dev, peaks):
                 "gbs_2": rate(out["hbm_2streams"]), "gbs_4": rate(out["hbm_4streams"]),
                 "frac_2": rate(out["hbm_2streams"]) / peaks["hbm_gbs"],
                 "frac_4": rate(out["hbm_4streams"]) / peaks["hbm_gbs"]},
-            "roofline": {"bound": "hbm", "kernel": "gemv_decode_kernel", "achieved": gbs, "peak": peaks["hbm_gbs"],
-                         "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC["gemv_decode_kernel"],
+            "roofline": {"bound": "hbm", "kernel": "gemv_decode_fast_kernel", "achieved": gbs, "peak": peaks["hbm_gbs"],
+                         "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC["gemv_decode_fast_kernel"],
                          "frac_of_nominal": gbs / NOMINAL_HBM_GBS, "peak_source": peaks["source"] + " copy"}}
 
 
@@ -539,9 +540,9 @@ def bench_pack(B, synth, dev, peaks):
     gbs = nbytes / (ms * 1e-3) / 1e9
     return {"workload": "binarize+pack W fp32 [4096,4096] -> 1 bit/weight (PREFILL layout), alpha, beta, rowsum",
             "ms": ms, "gpu_launches": 2 * reps,
-            "roofline": {"bound": "hbm", "kernel": "reduce_partials + sign_pack", "achieved": gbs,
+            "roofline": {"bound": "hbm", "kernel": "reduce_partials + sign_pack_rows", "achieved": gbs,
                          "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
-                         "traffic": NCU_TRAFFIC["reduce_partials + sign_pack"],
+                         "traffic": NCU_TRAFFIC["reduce_partials + sign_pack_rows"],
                          "peak_source": peaks["source"] + " copy"}}
 
 
@@ -791,8 +792,8 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
-    ap.add_argument("--parts", default="decode,pack,grouped,block,small,cpu",
-                    help="extra measurements beside the prefill step (comma list of decode, pack, grouped, block, small, cpu; "
+    ap.add_argument("--parts", default="calib,decode,pack,grouped,block,small,cpu",
+                    help="extra measurements beside the prefill step (comma list of calib, decode, pack, grouped, block, small, cpu; "
                          "'none' for the prefill step alone, e.g. under a profiler)")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
