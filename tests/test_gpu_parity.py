@@ -505,6 +505,35 @@ def test_gemv_decode(K, N, G, dtype, mode, relu):
     assert torch.equal(y16, y32.to(DT[dtype]))
 
 
+def test_gemv_decode_exact_ties_go_to_the_even_neighbour():
+    # Eta form with inputs on a coarse grid: x = j / 64 for integer j in [0, 256], min 0 and max 4,
+    # so (x - eta) Q_b / gamma = x * 32 = j / 2 is an exact half-integer for every odd j.  The decode
+    # kernel settles such elements in exact arithmetic (Eq. 6 with round-half-to-even), so its
+    # codes are known without running anything: rne(j / 2) clipped to 127.  The oracle's matmul and
+    # rescale on those codes give y; no code may differ, so the plain tolerance applies.
+    K, N = 4096, 256
+    rng = np.random.default_rng(3)
+    j = rng.integers(0, 257, size=K)
+    j[0], j[1] = 0, 256
+    x = torch.tensor(j / 64.0, dtype=torch.float16).reshape(1, K)
+    assert (x.double().numpy()[0] * 64 == j).all()                      # exactly representable
+    half = j // 2
+    codes = np.where(j % 2 == 0, half, half + (half % 2)).clip(0, 127).astype(np.int8).reshape(1, K)
+    assert np.count_nonzero(j % 2) > K // 3                             # ties everywhere
+    W = synth.make_w(N, K, torch.float32, seed=9)
+    w_ref = O.binarize(W.numpy())
+    w_gpu = B.binarize_pack(W.to(DEV), layout=B.DECODE)
+    torch.cuda.synchronize()
+    q_ref = O.quant_act(x.float().numpy(), mode=O.ETA, gran=O.PER_TOKEN, ln_eps=1e-5)   # for gamma only
+    acc = O.matmul(codes, w_ref["bits"])
+    want = O.dequant(acc, w_ref["beta"], q_ref["gamma"], gran=O.PER_TOKEN)[0]
+    y = B.gemv_decode(x.to(DEV), w_gpu["W_packed"], w_gpu["beta"], N, mode=B.ETA, ln_eps=1e-5,
+                      out_dtype=torch.float32)
+    torch.cuda.synchronize()
+    rms = np.sqrt((want ** 2).mean())
+    assert np.abs(y.cpu().numpy().astype(np.float64) - want).max() <= FLOAT_TOL_RMS * rms
+
+
 def test_gemv_decode_weights_from_global_memory_when_the_wait_runs_out():
     # With the poll limit of the kernel's one bounded wait at zero, warps whose weight stage has not
     # landed at their first look read it from global memory instead: same bits, same y.
