@@ -279,10 +279,13 @@ bl_status bitlinear_gemv_decode(const void* x, bl_dtype xt, int64_t K, int64_t N
  * per-token inference of Sec. 2.1 with one weight stream shared by the batch).  Each token gets
  * its own LN statistics, gamma and eta (Eq. 12, 4-6 per token); up to 8 tokens share one pass
  * over the packed weights (tensor-core mma on bit planes of the packed words), larger M runs
- * ceil(M/8) passes with the weights served from L2.
+ * ceil(M/8) passes with the weights served from L2.  For M >= 2 a token's result does not depend on
+ * what else is in the batch (same bits); M == 1 is handed to the kernel of bitlinear_gemv_decode,
+ * which is faster for one token and may differ from this one in the last bit of gamma.  W_packed
+ * is read ahead of stream order, as there.
  *   x [M,K] of dtype xt;  y [M,N] of dtype yt;  W_packed in DECODE layout.
  *   K % 256 == 0, (K/G) % 256 == 0, N % 16 == 0, min(M, 8) * (K + 16) <= 155 KB (BL_ERR_SHAPE otherwise).
- * No workspace, no device-side waits. */
+ * No workspace; no device-side waits for M >= 2. */
 bl_status bitlinear_gemv_decode_batch(const void* x, bl_dtype xt, int64_t M, int64_t K, int64_t N, int G,
                                       int b, bl_quant_mode mode, float ln_eps, int eta_correction,
                                       const uint8_t* W_packed, const float* beta, const int32_t* rowsum,

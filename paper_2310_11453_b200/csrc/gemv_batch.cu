@@ -383,8 +383,11 @@ bool gemv_batch_supported(int64_t M, int64_t K, int64_t N, int G) {
          batch_smem(M < kBatchTokens ? M : kBatchTokens, K, 0, false) <= kSmemBudget;
 }
 
-// M tokens in launches of up to 8; later launches find the weights in L2.
+// M tokens in launches of up to 8; later launches find the weights in L2.  A single token goes to the
+// single-token kernel (half the time of this one at M = 1; its statistics are summed in another order,
+// so its gamma may differ from this kernel's in the last bit).
 cudaError_t launch_gemv_batch(const GemvArgs& g, int64_t M, cudaStream_t s) {
+  if (M == 1 && g.K <= 32768) return launch_gemv_decode(g, s);
   const size_t xsz = g.xt == BL_F32 ? 4 : 2, ysz = g.yt == BL_F32 ? 4 : 2;
   for (int64_t m0 = 0; m0 < M; m0 += kBatchTokens) {
     BatchArgs a;

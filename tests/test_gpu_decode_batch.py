@@ -65,11 +65,18 @@ def test_gemv_decode_batch(M, K, N, G, dtype, mode, relu):
     if dtype != "f32":
         y16 = B.gemv_decode_batch(xd, w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode, out_dtype=DT[dtype])
         assert torch.equal(y16, y32.to(DT[dtype]))
-    # a token's result does not depend on what else is in the batch
+    # a token's result does not depend on what else is in the batch: the last two tokens as a batch of
+    # their own give the same bits (a single token takes the single-token kernel, whose sums run in
+    # another order: same codes up to the tolerated ties, gamma to the last bit or so)
+    if M > 2:
+        y_two = B.gemv_decode_batch(xd[M - 2:M].contiguous(), w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode,
+                                    out_dtype=torch.float32)
+        assert torch.equal(y_two, y32[M - 2:M])
     if M > 1:
         y_one = B.gemv_decode_batch(xd[M - 1:M].contiguous(), w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode,
                                     out_dtype=torch.float32)
-        assert torch.equal(y_one[0], y32[M - 1])
+        d = np.abs(y_one[0].cpu().numpy().astype(np.float64) - y32[M - 1].cpu().numpy().astype(np.float64))
+        assert (d <= 1e-3 * rms + slack[M - 1]).all()
 
 
 def test_gemv_decode_batch_integer_definition_exactly():
