@@ -496,6 +496,48 @@ def bench_decode(B, synth, dev, peaks):
                            "weight_gbs": (N * K / 8 + Mb * 2 * (K + N)) / (us * 1e-6) / 1e9}
         del graph
 
+    # the same call on projection shapes of the larger models of the paper's Table 1 sizes
+    del packs, y, yb
+    other = {}
+    ocalls = 200
+    for label, Ko, No in (("6.7B FFN down", 16384, 4096), ("13B FFN up", 5120, 20480), ("30B attention", 7168, 7168)):
+        obufs = -(-(256 << 20) // (No * Ko // 8))            # 256 MiB of packed weights in rotation
+        opacks = []
+        for _ in range(obufs):
+            Wd = torch.randn((No, Ko), generator=gen, device=dev, dtype=torch.float32) * synth.W_STD
+            opacks.append(B.binarize_pack(Wd, layout=B.DECODE, want_rowsum=False))
+            del Wd
+        torch.cuda.synchronize()
+        xo = synth.make_x(ocalls, Ko, torch.float16, seed=3, outliers=False).to(dev)
+        yo = torch.empty((ocalls, No), dtype=torch.float16, device=dev)
+
+        def issue_other():
+            for i in range(ocalls):
+                p = opacks[i % obufs]
+                B.gemv_decode(xo[i], p["W_packed"], p["beta"], No, y=yo[i])
+        issue_other()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            issue_other()
+        for _ in range(2):
+            graph.replay()
+        torch.cuda.synchronize()
+        times = []
+        for _ in range(5):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            graph.replay()
+            b.record()
+            torch.cuda.synchronize()
+            times.append(a.elapsed_time(b))
+        us = statistics.median(times) / ocalls * 1e3
+        ob = No * Ko / 8 + 2 * Ko + 2 * No
+        other[label] = {"K": Ko, "N": No, "us_per_call": us, "gbs": ob / (us * 1e-6) / 1e9,
+                        "frac": ob / (us * 1e-6) / 1e9 / peaks["hbm_gbs"]}
+        del graph, opacks, xo, yo
+    fallbacks = B.debug_decode_fallbacks()
+
     def rate(us):
         return bytes_per_call / (us * 1e-6) / 1e9
 
@@ -504,6 +546,8 @@ def bench_decode(B, synth, dev, peaks):
                         "(every call ordered after the one before it)",
             "us_per_call": out["hbm"], "us_per_call_l2_hot": out["l2_hot"], "bytes_per_call": bytes_per_call,
             "gpu_launches": calls,
+            "other_shapes": {"note": "one stream, 200 calls in one CUDA graph rotating over 256 MiB of weight buffers", **other},
+            "waits_run_out": fallbacks,
             "small_batch": {"note": "bitlinear_gemv_decode_batch, M tokens per call (one launch per 8 tokens), "
                                     "400 calls in one CUDA graph over the same 64 weight buffers, one stream",
                             **batch},

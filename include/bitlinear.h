@@ -341,13 +341,21 @@ bl_status bitlinear_ws_status(const void* ws, void* stream);
 /* Test and diagnostic hook: caps the number of polls that the bounded device-side waits of
  * kernels launched afterwards by this process may make (bitlinear_gemv_decode's wait for its
  * weight copies; the meeting between the two passes of the cooperative per-tensor kernel of
- * bitlinear_quant_act).  polls < 0 restores the built-in limits; 0 means a single poll.
+ * bitlinear_quant_act).  polls < 0 restores the built-in limits; 0 means a single poll (for
+ * bitlinear_gemv_decode: none at all, every warp reads its weights from global memory).
  * meet_skew != 0 additionally makes the cooperative kernel wait for an arrival tag that no CTA
  * publishes, so that its wait runs out by construction: the kernel then records
  * BL_ERR_TIMEOUT in the status word, writes no codes and returns (nothing hangs, traps or
  * faults).  Process-wide and not synchronised with calls in flight on other host threads; not for
  * production use.  Always returns BL_OK. */
 bl_status bitlinear_debug_wait_limit(int64_t polls, int meet_skew);
+
+/* Test and diagnostic hook: synchronises `stream`, then returns and clears the number of warps of
+ * bitlinear_gemv_decode kernels (on the current device, since the last call of this function) whose
+ * bounded wait for a stage of weights ran out, so that they read the stage from global memory
+ * instead.  The result of such a call is still correct, only slow; a healthy run returns 0.
+ * -1 on a CUDA error. */
+int64_t bitlinear_debug_decode_fallbacks(void* stream);
 
 #ifdef __cplusplus
 }

@@ -30,7 +30,7 @@ EXPORTS = [
     "bitlinear_forward", "bitlinear_matmul_i32", "bitlinear_matmul_dequant", "bitlinear_gemv_decode",
     "bitlinear_attention_causal", "bitlinear_block_forward", "bitlinear_ws_status",
     "bitlinear_matmul_dequant_ex", "bitlinear_binarize_pack_nsplit", "bitlinear_gemv_decode_batch",
-    "bitlinear_forward_latent", "bitlinear_debug_wait_limit", "bitlinear_noalloc_status",
+    "bitlinear_forward_latent", "bitlinear_debug_wait_limit", "bitlinear_noalloc_status", "bitlinear_debug_decode_fallbacks",
 ]
 
 _DTYPES = {torch.float32: F32, torch.float16: F16, torch.bfloat16: BF16}
@@ -94,6 +94,8 @@ def lib():
                                                   ci, vp]
         L.bitlinear_binarize_pack_nsplit.restype = ci
         L.bitlinear_binarize_pack_nsplit.argtypes = [vp, ci, i64, i64, ci, ci, ci, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.bitlinear_debug_decode_fallbacks.restype = i64
+        L.bitlinear_debug_decode_fallbacks.argtypes = [vp]
         L.bitlinear_noalloc_status.restype = ci
         L.bitlinear_noalloc_status.argtypes = [vp]
         L.bitlinear_debug_wait_limit.restype = ci
@@ -400,6 +402,11 @@ def block_forward(x, weights, batch, seq, heads, ffn, ln_eps=1e-5, ws=None, fuse
     _check(code, "bitlinear_block_forward")
     out["ws"] = ws
     return out
+
+
+def debug_decode_fallbacks() -> int:
+    """bitlinear_debug_decode_fallbacks: synchronises; warps that read weights from global memory since the last call."""
+    return int(lib().bitlinear_debug_decode_fallbacks(_stream()))
 
 
 def noalloc_status() -> int:

@@ -473,6 +473,13 @@ bl_status bitlinear_ws_status(const void* ws, void* stream) {
   return word == 0 ? BL_OK : BL_ERR_TIMEOUT;
 }
 
+int64_t bitlinear_debug_decode_fallbacks(void* stream) {
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return -1;
+  unsigned int n = 0;
+  if (gemv_decode_take_fallbacks(&n) != cudaSuccess) return -1;
+  return (int64_t)n;
+}
+
 bl_status bitlinear_debug_wait_limit(int64_t polls, int meet_skew) {
   g_debug_wait_polls.store(polls < 0 ? -1 : (long long)polls, std::memory_order_relaxed);
   g_debug_meet_skew.store(meet_skew ? 1 : 0, std::memory_order_relaxed);

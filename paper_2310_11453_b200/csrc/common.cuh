@@ -190,6 +190,7 @@ struct GemvArgs {
   void* y; bl_dtype yt;
 };
 cudaError_t launch_gemv_decode(const GemvArgs& a, cudaStream_t s);
+cudaError_t gemv_decode_take_fallbacks(unsigned int* out);   // warps that read weights from global memory after a wait ran out
 // The same for M tokens (x [M,K], y [M,N]) sharing one pass over the weights per 8 tokens.
 cudaError_t launch_gemv_batch(const GemvArgs& a, int64_t M, cudaStream_t s);
 bool gemv_batch_supported(int64_t M, int64_t K, int64_t N, int G);

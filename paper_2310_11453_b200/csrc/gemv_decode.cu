@@ -159,6 +159,8 @@ __device__ __forceinline__ void accumulate8(const float (&v)[8], float& s1, floa
 }
 
 // ---- ring of weight stages ---------------------------------------------------------------------------
+__device__ unsigned int g_fallbacks;          // warps whose wait for a weight stage ran out (since last read)
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ bool bar_poll(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -192,7 +194,7 @@ struct GemvGeom {            // decided on the host
   int depth;                 // ring slots in use (<= kMaxStages)
   uint32_t stage_stride;     // bytes between ring slots (a multiple of 128)
   uint32_t ring_bytes;       // depth * stage_stride
-  uint32_t wait_polls;       // polls of a stage barrier before the warp falls back to global loads
+  uint32_t wait_polls;       // polls of a stage barrier before the warp falls back to global loads (0: at once)
   uint32_t inv_nslices, inv_group_chunks;   // ceil(2^16 / d): (v * inv) >> 16 == v / d for v < 256
   double inv_kg;
 };
@@ -208,11 +210,14 @@ gemv_decode_kernel(GemvArgs a, GemvGeom geo) {
   const int K = (int)a.K, G = a.G, Kg = K / G;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t Kb = a.K / 8;
-  const int rpw = geo.rpw, nstages = geo.nstages, nslices = geo.nslices, rowslots = geo.rowslots, depth = geo.depth;
+  const int rpw = geo.rpw, nslices = geo.nslices, rowslots = geo.rowslots, depth = geo.depth;
   const int stage_rows = rpw * rowslots;
   const int64_t row_begin = (int64_t)blockIdx.x * geo.rows_per_cta;
   const int64_t row_end = min((int64_t)a.N, row_begin + geo.rows_per_cta);
   const int rows_cta = (int)(row_end - row_begin);
+  // stages that hold rows of this CTA (the last CTA has fewer rows than the others): a stage without
+  // rows gets no copy, so nobody may wait for one
+  const int nstages = min(geo.nstages, (rows_cta + stage_rows - 1) / stage_rows);
   const uint8_t* wslice = a.W_packed + row_begin * Kb;
 
   // Copy of stage st into its ring slot; called by one thread once every reader of the slot's
@@ -445,9 +450,9 @@ gemv_decode_kernel(GemvArgs a, GemvGeom geo) {
     const int slot = st % depth;
     if (!from_global) {
       if (*reinterpret_cast<volatile int*>(&sh.abandon)) from_global = true;
-      else if (!bar_wait(smem_u32(&sh.full[slot]), (uint32_t)(st / depth) & 1u, geo.wait_polls)) {
+      else if (geo.wait_polls == 0 || !bar_wait(smem_u32(&sh.full[slot]), (uint32_t)(st / depth) & 1u, geo.wait_polls)) {
         from_global = true;
-        if (lane == 0) { atomicExch(&sh.abandon, 1); __threadfence_block(); }
+        if (lane == 0) { atomicExch(&sh.abandon, 1); __threadfence_block(); atomicAdd(&g_fallbacks, 1u); }
       }
     }
     if (st == 0) BL_STAMP(8);
@@ -548,7 +553,8 @@ gemv_decode_kernel(GemvArgs a, GemvGeom geo) {
 
 
 // ====================================================================================================
-// The common case: one group, K a multiple of 4096, Eq. 11 as printed (no row terms).
+// The common case: one group, Eq. 11 as printed (no row terms).  K is taken in slices of 4096; the
+// last one may be partial.
 //
 // Measured on this kernel family: every instruction of a call runs only a handful of times, two
 // warps per scheduler hide little, and a conditional branch inside the row loop costs more than the
@@ -611,7 +617,7 @@ __device__ __forceinline__ void warp_rows(const uint32_t (&xr)[32], int rpw, uin
   }
 }
 
-// kSingle: K == 4096.  The thread's 16 features then stay in registers between the two passes, no
+// kSingle: K <= 4096 (one slice).  The thread's 16 features then stay in registers between the two passes, no
 // raw copy of x is kept in shared memory, and three CTAs fit on an SM (the call in progress and two
 // calls staging their weights behind it, or three independent calls).
 template <typename TX, typename TY, bool kSingle>
@@ -620,16 +626,20 @@ gemv_decode_fast_kernel(GemvArgs a, FastGeom geo) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   __shared__ FastShared sh;
   unsigned char* ring = smem_raw;                                                  // [depth][stage_stride] (+ one row)
-  const uint32_t ring_alloc = geo.ring_bytes + (uint32_t)(a.K / 8);
-  float* xf = reinterpret_cast<float*>(smem_raw + ring_alloc);                     // [K] raw x (not for kSingle)
-  int8_t* codes = reinterpret_cast<int8_t*>(smem_raw + ring_alloc + (kSingle ? 0 : a.K * sizeof(float)));   // [K]
+  const int K = (int)a.K, Kp = geo.nslices * kSlice;                               // K rounded up to whole slices
+  const uint32_t ring_alloc = geo.ring_bytes + (uint32_t)(a.K / 8) + 512u;         // lanes of a partial slice read past a row's end
+  float* xf = reinterpret_cast<float*>(smem_raw + ring_alloc);                     // [Kp] raw x (not for kSingle)
+  int8_t* codes = reinterpret_cast<int8_t*>(smem_raw + ring_alloc + (kSingle ? 0 : (size_t)Kp * sizeof(float)));   // [Kp]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t Kb = a.K / 8;
-  const int rpw = geo.rpw, nstages = geo.nstages, nslices = geo.nslices, depth = geo.depth;
+  const int rpw = geo.rpw, nslices = geo.nslices, depth = geo.depth;
   const int stage_rows = rpw * kGemvWarps;
   const int64_t row_begin = (int64_t)blockIdx.x * geo.rows_per_cta;
   const int64_t row_end = min((int64_t)a.N, row_begin + geo.rows_per_cta);
   const int rows_cta = (int)(row_end - row_begin);
+  // stages that hold rows of this CTA (the last CTA has fewer rows than the others): a stage without
+  // rows gets no copy, so nobody may wait for one
+  const int nstages = min(geo.nstages, (rows_cta + stage_rows - 1) / stage_rows);
   const uint8_t* wslice = a.W_packed + row_begin * Kb;
 
   auto issue_stage = [&](int st, int slot) {
@@ -678,21 +688,26 @@ gemv_decode_fast_kernel(GemvArgs a, FastGeom geo) {
   // ---- x: 16 features per thread and slice, sums around the pilot, raw values to shared memory -------
   const TX* x = reinterpret_cast<const TX*>(a.x);
   const float beta = __ldg(a.beta);
-  float pilot;
+  float pilot, fill;                                    // fill: a real feature, standing in for absent ones in min / max
   {
     float h[8];
     Elem<TX>::load8(x, h);
     pilot = (((h[0] + h[1]) + (h[2] + h[3])) + ((h[4] + h[5]) + (h[6] + h[7]))) * 0.125f;
+    fill = h[0];
   }
   const bool ln = a.ln_eps >= 0.f;
   if (!ln) pilot = 0.f;
   float s1 = 0.f, s2 = 0.f, mn = INFINITY, mx = -INFINITY;
   float xv[16];                                         // kSingle: this thread's features
+  // Features past K (K need not fill its last slice of 4096) are absent: they add nothing to the
+  // sums, stand as `fill` in the extremes, get code 0, and the lanes that own them multiply zeros.
   // sums of 16 raw features around the pilot, and their extremes
-  auto moments16 = [&](const float (&v)[16]) {
+  auto moments16 = [&](int i, const float (&v)[16]) {
+    const int k = i * kSlice + threadIdx.x * 8;
+    const bool have[2] = {k < K, k + kSlice / 2 < K};
     float d[16];
 #pragma unroll
-    for (int j = 0; j < 16; ++j) { d[j] = v[j] - pilot; mn = fminf(mn, v[j]); mx = fmaxf(mx, v[j]); }
+    for (int j = 0; j < 16; ++j) { d[j] = have[j >> 3] ? v[j] - pilot : 0.f; mn = fminf(mn, v[j]); mx = fmaxf(mx, v[j]); }
     s1 += (((d[0] + d[1]) + (d[2] + d[3])) + ((d[4] + d[5]) + (d[6] + d[7]))) +
           (((d[8] + d[9]) + (d[10] + d[11])) + ((d[12] + d[13]) + (d[14] + d[15])));
     float p2 = 0.f, q2 = 0.f;
@@ -704,14 +719,16 @@ gemv_decode_fast_kernel(GemvArgs a, FastGeom geo) {
   auto load16 = [&](int i, float (&v)[16]) {
     const int k = i * kSlice + threadIdx.x * 8;
     float lo8[8], hi8[8];
-    Elem<TX>::load8(x + k, lo8);
-    Elem<TX>::load8(x + k + kSlice / 2, hi8);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { lo8[j] = fill; hi8[j] = fill; }
+    if (k < K) Elem<TX>::load8(x + k, lo8);
+    if (k + kSlice / 2 < K) Elem<TX>::load8(x + k + kSlice / 2, hi8);
 #pragma unroll
     for (int j = 0; j < 8; ++j) { v[j] = lo8[j]; v[8 + j] = hi8[j]; }
   };
   if (kSingle) {
     load16(0, xv);
-    moments16(xv);
+    moments16(0, xv);
   } else {
 #pragma unroll 1
     for (int i = 0; i < nslices; ++i) {
@@ -723,7 +740,7 @@ gemv_decode_fast_kernel(GemvArgs a, FastGeom geo) {
         *reinterpret_cast<float4*>(xf + k + h * (kSlice / 2)) = make_float4(v[8 * h], v[8 * h + 1], v[8 * h + 2], v[8 * h + 3]);
         *reinterpret_cast<float4*>(xf + k + h * (kSlice / 2) + 4) = make_float4(v[8 * h + 4], v[8 * h + 5], v[8 * h + 6], v[8 * h + 7]);
       }
-      moments16(v);
+      moments16(i, v);
     }
   }
   BL_STAMP(3);
@@ -786,8 +803,9 @@ gemv_decode_fast_kernel(GemvArgs a, FastGeom geo) {
     }
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-      const uint32_t w0 = __byte_perm(__byte_perm(tb[8 * h], tb[8 * h + 1], 0x0040), __byte_perm(tb[8 * h + 2], tb[8 * h + 3], 0x0040), 0x5410);
-      const uint32_t w1 = __byte_perm(__byte_perm(tb[8 * h + 4], tb[8 * h + 5], 0x0040), __byte_perm(tb[8 * h + 6], tb[8 * h + 7], 0x0040), 0x5410);
+      uint32_t w0 = __byte_perm(__byte_perm(tb[8 * h], tb[8 * h + 1], 0x0040), __byte_perm(tb[8 * h + 2], tb[8 * h + 3], 0x0040), 0x5410);
+      uint32_t w1 = __byte_perm(__byte_perm(tb[8 * h + 4], tb[8 * h + 5], 0x0040), __byte_perm(tb[8 * h + 6], tb[8 * h + 7], 0x0040), 0x5410);
+      if (k + h * (kSlice / 2) >= K) { w0 = 0u; w1 = 0u; }              // absent features
       *reinterpret_cast<uint2*>(codes + code_slot(k + h * (kSlice / 2))) = make_uint2(w0, w1);
       csum = __dp4a((int)w0, 0x01010101, csum);
       csum = __dp4a((int)w1, 0x01010101, csum);
@@ -854,20 +872,20 @@ gemv_decode_fast_kernel(GemvArgs a, FastGeom geo) {
   for (int st = 0; st < nstages; ++st) {
     if (!from_global) {
       if (*reinterpret_cast<volatile int*>(&sh.abandon)) from_global = true;
-      else if (!bar_wait(smem_u32(&sh.full[slot]), phase, geo.wait_polls)) {
+      else if (geo.wait_polls == 0 || !bar_wait(smem_u32(&sh.full[slot]), phase, geo.wait_polls)) {
         from_global = true;
-        if (lane == 0) { atomicExch(&sh.abandon, 1); __threadfence_block(); }
+        if (lane == 0) { atomicExch(&sh.abandon, 1); __threadfence_block(); atomicAdd(&g_fallbacks, 1u); }
       }
     }
     if (st == 0) BL_STAMP(9);
     const int row0 = st * stage_rows + warp * rpw;      // first row of this warp in the stage (CTA-local)
     const int rows_left = rows_cta - row0;              // may be <= 0: nothing of this warp is stored
     const uint32_t wsm = slot_addr + warp_off;
-    const uint8_t* wgl = wslice + (int64_t)min(row0, rows_cta - 1) * Kb + lane * 16;   // only read after a failed wait
+    const uint8_t* wgl = wslice + (int64_t)min(row0, rows_cta - 1) * Kb;               // only read after a failed wait
     const int rl = max(rows_left, 1);
     if (kSingle) {
       if (!from_global) warp_rows<true, false>(xr, rpw, wsm, wgl, Kb, rl, acc_lane);
-      else warp_rows<true, true>(xr, rpw, wsm, wgl, Kb, rl, acc_lane);
+      else warp_rows<true, true>(xr, rpw, wsm, wgl + min((int64_t)lane * 16, Kb - 16), Kb, rl, acc_lane);
     } else {
 #pragma unroll 1
       for (int s = 0; s < nslices; ++s) {
@@ -876,8 +894,10 @@ gemv_decode_fast_kernel(GemvArgs a, FastGeom geo) {
           if (s == 0) warp_rows<true, false>(xr, rpw, wsm, wgl, Kb, rl, acc_lane);
           else warp_rows<false, false>(xr, rpw, wsm + s * 512, wgl, Kb, rl, acc_lane);
         } else {
-          if (s == 0) warp_rows<true, true>(xr, rpw, wsm, wgl, Kb, rl, acc_lane);
-          else warp_rows<false, true>(xr, rpw, wsm, wgl + s * 512, Kb, rl, acc_lane);
+          // (a lane whose chunk lies past K multiplies zero codes: any bytes of the row will do)
+          const uint8_t* wl = wgl + min((int64_t)s * 512 + lane * 16, Kb - 16);
+          if (s == 0) warp_rows<true, true>(xr, rpw, wsm, wl, Kb, rl, acc_lane);
+          else warp_rows<false, true>(xr, rpw, wsm, wl, Kb, rl, acc_lane);
         }
       }
     }
@@ -930,7 +950,7 @@ template <typename TX, typename TY>
 cudaError_t run_fast(const GemvArgs& a, cudaStream_t s, int dev, int sms) {
   FastGeom geo;
   const int64_t Kb = a.K / 8;
-  geo.nslices = (int)(a.K / kSlice);
+  geo.nslices = (int)((a.K + kSlice - 1) / kSlice);
   const int64_t rows_per_cta = (a.N + sms - 1) / sms;
   const int64_t per_warp = (rows_per_cta + kGemvWarps - 1) / kGemvWarps;
   const int64_t rmax = std::max<int64_t>(1, std::min<int64_t>(kBatchRows, 32768 / (kGemvWarps * Kb)));
@@ -941,7 +961,8 @@ cudaError_t run_fast(const GemvArgs& a, cudaStream_t s, int dev, int sms) {
   geo.rpw = (int)((per_warp + nstages - 1) / nstages);
   geo.stage_stride = (uint32_t)(geo.rpw * kGemvWarps * Kb);                      // a multiple of 4096, at most 32 KB
   const bool single = geo.nslices == 1;
-  const size_t fixed = (size_t)a.K * (single ? 1 : sizeof(float) + 1) + (size_t)Kb;   // (raw x,) codes, one row beyond the ring
+  const size_t Kp = (size_t)geo.nslices * kSlice;
+  const size_t fixed = Kp * (single ? 1 : sizeof(float) + 1) + (size_t)Kb + 512;   // (raw x,) codes, slack beyond the ring
   const size_t budget = std::min<size_t>(kRingBytes, 210 * 1024 - fixed);
   const int depth = std::max(1, std::min((int)(budget / geo.stage_stride), kMaxStages));
   geo.depth = (int)std::min<int64_t>(depth, nstages);
@@ -984,7 +1005,7 @@ cudaError_t run2(const GemvArgs& a, cudaStream_t s) {
   if (e != cudaSuccess) return e;
   e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
-  if (a.G == 1 && a.K % kSlice == 0 && !a.eta_correction) return run_fast<TX, TY>(a, s, dev, sms);
+  if (a.G == 1 && !a.eta_correction) return run_fast<TX, TY>(a, s, dev, sms);
   // One CTA per SM when there are enough rows; every row slot takes its rows in stages of at most
   // kBatchRows, all stages the same height.
   GemvGeom geo;
@@ -1049,6 +1070,18 @@ cudaError_t run1(const GemvArgs& a, cudaStream_t s) {
 }
 
 }  // namespace
+
+// Reads and clears the count of warps that gave up waiting for a weight stage and read it from
+// global memory instead.
+cudaError_t gemv_decode_take_fallbacks(unsigned int* out) {
+  cudaError_t e = cudaMemcpyFromSymbol(out, g_fallbacks, sizeof(unsigned int));
+  if (e != cudaSuccess) return e;
+  if (*out) {
+    const unsigned int zero = 0;
+    e = cudaMemcpyToSymbol(g_fallbacks, &zero, sizeof(zero));
+  }
+  return e;
+}
 
 cudaError_t launch_gemv_decode(const GemvArgs& a, cudaStream_t s) {
   switch (a.xt) {

@@ -470,6 +470,11 @@ def explained_by_code_flips(err, signs, step, tol, max_flips):
     (4096, 16384, 1, "bf16", "eta", True),         # c2-shaped, eta form (with and without the row terms)
     (12288, 4096, 1, "f16", "absmax", False),      # three slices per row
     (4096, 160000, 1, "f16", "absmax", False),     # 1082 rows per CTA: the ring is refilled many times
+    (5120, 1024, 1, "bf16", "absmax", False),      # 13B-shaped width: a whole slice and a quarter of one
+    (768, 3072, 1, "f32", "absmax", False),        # 125M-shaped width: a partial slice only
+    (7168, 512, 1, "f16", "eta", True),            # 30B-shaped width, eta form
+    (16384, 4096, 1, "f16", "absmax", False),      # the last CTA has rows in the first of its two stages only
+    (1024, 4000 * 16, 2, "bf16", "eta", True),     # the same in the kernel for groups
 ])
 def test_gemv_decode(K, N, G, dtype, mode, relu):
     x = synth.make_x(1, K, DT[dtype], seed=K + N, outliers=False, relu=relu)
@@ -503,6 +508,9 @@ def test_gemv_decode(K, N, G, dtype, mode, relu):
     y32 = B.gemv_decode(x.to(DEV), w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode, ln_eps=1e-5,
                         out_dtype=torch.float32)
     assert torch.equal(y16, y32.to(DT[dtype]))
+    # every stage of weights arrived through its copy: no warp had to fall back to global loads (a
+    # stage that is waited for but never copied would still give the right y, a second late per call)
+    assert B.debug_decode_fallbacks() == 0
 
 
 def test_gemv_decode_exact_ties_go_to_the_even_neighbour():
@@ -535,19 +543,20 @@ def test_gemv_decode_exact_ties_go_to_the_even_neighbour():
 
 
 def test_gemv_decode_weights_from_global_memory_when_the_wait_runs_out():
-    # With the poll limit of the kernel's one bounded wait at zero, warps whose weight stage has not
-    # landed at their first look read it from global memory instead: same bits, same y.
+    # With the poll limit of the kernel's one bounded wait at zero every warp takes its wait to have run
+    # out and reads its weights from global memory instead: same bits, same y.
     for K, N in [(4096, 16384), (1024, 40960), (8192, 2048)]:
         x = synth.make_x(1, K, torch.float16, seed=K, outliers=False).to(DEV)
         w = B.binarize_pack(synth.make_w(N, K, torch.float32, seed=K + 1).to(DEV), layout=B.DECODE)
         torch.cuda.synchronize()
         want = B.gemv_decode(x, w["W_packed"], w["beta"], N, out_dtype=torch.float32)
+        assert B.debug_decode_fallbacks() == 0
         try:
             B.debug_wait_limit(0)
             got = [B.gemv_decode(x, w["W_packed"], w["beta"], N, out_dtype=torch.float32) for _ in range(3)]
         finally:
             B.debug_wait_limit(-1)
-        torch.cuda.synchronize()
+        assert B.debug_decode_fallbacks() >= 3 * 8       # every warp of every CTA took the other path
         for g in got:
             assert torch.equal(g, want)
 
