@@ -620,7 +620,8 @@ __device__ __forceinline__ void warp_rows(const uint32_t (&xr)[32], int rpw, uin
 // kSingle: K <= 4096 (one slice).  The thread's 16 features then stay in registers between the two passes, no
 // raw copy of x is kept in shared memory, and three CTAs fit on an SM (the call in progress and two
 // calls staging their weights behind it, or three independent calls).
-template <typename TX, typename TY, bool kSingle>
+// kPartial: K does not fill its last slice; only then does the code test features for presence.
+template <typename TX, typename TY, bool kSingle, bool kPartial>
 __global__ void __launch_bounds__(kGemvThreads, kSingle ? 3 : 2)
 gemv_decode_fast_kernel(GemvArgs a, FastGeom geo) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -688,23 +689,22 @@ gemv_decode_fast_kernel(GemvArgs a, FastGeom geo) {
   // ---- x: 16 features per thread and slice, sums around the pilot, raw values to shared memory -------
   const TX* x = reinterpret_cast<const TX*>(a.x);
   const float beta = __ldg(a.beta);
-  float pilot, fill;                                    // fill: a real feature, standing in for absent ones in min / max
+  float pilot;
   {
     float h[8];
     Elem<TX>::load8(x, h);
     pilot = (((h[0] + h[1]) + (h[2] + h[3])) + ((h[4] + h[5]) + (h[6] + h[7]))) * 0.125f;
-    fill = h[0];
   }
   const bool ln = a.ln_eps >= 0.f;
   if (!ln) pilot = 0.f;
   float s1 = 0.f, s2 = 0.f, mn = INFINITY, mx = -INFINITY;
   float xv[16];                                         // kSingle: this thread's features
   // Features past K (K need not fill its last slice of 4096) are absent: they add nothing to the
-  // sums, stand as `fill` in the extremes, get code 0, and the lanes that own them multiply zeros.
+  // sums, are read as copies of real features for the extremes, get code 0, and the lanes that own them multiply zeros.
   // sums of 16 raw features around the pilot, and their extremes
   auto moments16 = [&](int i, const float (&v)[16]) {
     const int k = i * kSlice + threadIdx.x * 8;
-    const bool have[2] = {k < K, k + kSlice / 2 < K};
+    const bool have[2] = {!kPartial || k < K, !kPartial || k + kSlice / 2 < K};
     float d[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) { d[j] = have[j >> 3] ? v[j] - pilot : 0.f; mn = fminf(mn, v[j]); mx = fmaxf(mx, v[j]); }
@@ -719,10 +719,9 @@ gemv_decode_fast_kernel(GemvArgs a, FastGeom geo) {
   auto load16 = [&](int i, float (&v)[16]) {
     const int k = i * kSlice + threadIdx.x * 8;
     float lo8[8], hi8[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) { lo8[j] = fill; hi8[j] = fill; }
-    if (k < K) Elem<TX>::load8(x + k, lo8);
-    if (k + kSlice / 2 < K) Elem<TX>::load8(x + k + kSlice / 2, hi8);
+    // (absent features: the last eight real ones once more, which leaves the extremes alone)
+    Elem<TX>::load8(x + (kPartial ? min(k, K - 8) : k), lo8);
+    Elem<TX>::load8(x + (kPartial ? min(k + kSlice / 2, K - 8) : k + kSlice / 2), hi8);
 #pragma unroll
     for (int j = 0; j < 8; ++j) { v[j] = lo8[j]; v[8 + j] = hi8[j]; }
   };
@@ -805,7 +804,7 @@ gemv_decode_fast_kernel(GemvArgs a, FastGeom geo) {
     for (int h = 0; h < 2; ++h) {
       uint32_t w0 = __byte_perm(__byte_perm(tb[8 * h], tb[8 * h + 1], 0x0040), __byte_perm(tb[8 * h + 2], tb[8 * h + 3], 0x0040), 0x5410);
       uint32_t w1 = __byte_perm(__byte_perm(tb[8 * h + 4], tb[8 * h + 5], 0x0040), __byte_perm(tb[8 * h + 6], tb[8 * h + 7], 0x0040), 0x5410);
-      if (k + h * (kSlice / 2) >= K) { w0 = 0u; w1 = 0u; }              // absent features
+      if (kPartial && k + h * (kSlice / 2) >= K) { w0 = 0u; w1 = 0u; }              // absent features
       *reinterpret_cast<uint2*>(codes + code_slot(k + h * (kSlice / 2))) = make_uint2(w0, w1);
       csum = __dp4a((int)w0, 0x01010101, csum);
       csum = __dp4a((int)w1, 0x01010101, csum);
@@ -975,9 +974,12 @@ cudaError_t run_fast(const GemvArgs& a, cudaStream_t s, int dev, int sms) {
   const size_t smem = (size_t)geo.ring_bytes + fixed;
   static std::atomic<int> configured[64];
   cudaError_t e;
-  auto kern = single ? gemv_decode_fast_kernel<TX, TY, true> : gemv_decode_fast_kernel<TX, TY, false>;
+  const bool partial = a.K % kSlice != 0;
+  auto kern = single ? (partial ? gemv_decode_fast_kernel<TX, TY, true, true> : gemv_decode_fast_kernel<TX, TY, true, false>)
+                     : (partial ? gemv_decode_fast_kernel<TX, TY, false, true> : gemv_decode_fast_kernel<TX, TY, false, false>);
   if (dev >= 64 || !configured[dev].load(std::memory_order_acquire)) {
-    for (auto k : {gemv_decode_fast_kernel<TX, TY, true>, gemv_decode_fast_kernel<TX, TY, false>}) {
+    for (auto k : {gemv_decode_fast_kernel<TX, TY, true, true>, gemv_decode_fast_kernel<TX, TY, true, false>,
+                   gemv_decode_fast_kernel<TX, TY, false, true>, gemv_decode_fast_kernel<TX, TY, false, false>}) {
       e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 216 * 1024);
       if (e != cudaSuccess) return e;
       e = cudaFuncSetAttribute(k, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
