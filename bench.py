@@ -466,15 +466,20 @@ def bench_decode(B, synth, dev, peaks):
     gbs = bytes_per_call / (out["hbm"] * 1e-6) / 1e9
 
     # small batches through bitlinear_gemv_decode_batch: M tokens share one pass over the weights
-    batch = {}
+    batch, batch_ws = {}, {}
     bcalls = 400
-    yb = torch.empty((16, N), dtype=torch.float16, device=dev)
-    for Mb in (1, 2, 4, 8, 16):
+    yb = torch.empty((32, N), dtype=torch.float16, device=dev)
+    wsb = torch.empty(B.workspace_bytes(B.OP_GEMV_DECODE_BATCH, 32, N, K, 1), dtype=torch.uint8, device=dev)
+    for Mb, with_ws in ((1, False), (2, False), (4, False), (8, False), (16, False),
+                        (2, True), (4, True), (8, True), (16, True), (32, True)):
         def issue_batch():
             for i in range(bcalls):
                 p = packs[i % nbuf]
                 r0 = (i * Mb) % (calls - Mb)
-                B.gemv_decode_batch(x[r0:r0 + Mb], p["W_packed"], p["beta"], N, y=yb[:Mb])
+                if with_ws:
+                    B.gemv_decode_batch_ws(x[r0:r0 + Mb], p["W_packed"], p["beta"], N, y=yb[:Mb], ws=wsb)
+                else:
+                    B.gemv_decode_batch(x[r0:r0 + Mb], p["W_packed"], p["beta"], N, y=yb[:Mb])
         issue_batch()
         torch.cuda.synchronize()
         graph = torch.cuda.CUDAGraph()
@@ -492,9 +497,11 @@ def bench_decode(B, synth, dev, peaks):
             torch.cuda.synchronize()
             times.append(a.elapsed_time(b))
         us = statistics.median(times) / bcalls * 1e3
-        batch[f"M{Mb}"] = {"us_per_call": us, "us_per_token": us / Mb,
-                           "weight_gbs": (N * K / 8 + Mb * 2 * (K + N)) / (us * 1e-6) / 1e9}
+        (batch_ws if with_ws else batch)[f"M{Mb}"] = {"us_per_call": us, "us_per_token": us / Mb,
+                                                      "weight_gbs": (N * K / 8 + Mb * 2 * (K + N)) / (us * 1e-6) / 1e9}
         del graph
+    if B.ws_status(wsb) != B.OK:
+        raise RuntimeError("a bounded wait of the tensor-core decode kernel ran out during the bench")
 
     # the same call on projection shapes of the larger models of the paper's Table 1 sizes
     del packs, y, yb
@@ -551,6 +558,9 @@ def bench_decode(B, synth, dev, peaks):
             "small_batch": {"note": "bitlinear_gemv_decode_batch, M tokens per call (one launch per 8 tokens), "
                                     "400 calls in one CUDA graph over the same 64 weight buffers, one stream",
                             **batch},
+            "small_batch_ws": {"note": "bitlinear_gemv_decode_batch_ws (workspace; a quantising kernel, then one tcgen05 "
+                                       "product kernel per 16 tokens), same graph and buffers",
+                               **batch_ws},
             "independent_streams": {
                 "note": "same 1000 calls spread round-robin over 2 / 4 streams inside the graph: calls on "
                         "different streams do not wait for one another",

@@ -83,7 +83,8 @@ typedef enum {
   BL_OP_MATMUL_I32 = 3,
   BL_OP_MATMUL_DEQUANT = 4,
   BL_OP_BLOCK_FORWARD = 5,   /* M = batch * seq tokens, N = ffn width, K = model width d, G ignored (1) */
-  BL_OP_FORWARD_LATENT = 6
+  BL_OP_FORWARD_LATENT = 6,
+  BL_OP_GEMV_DECODE_BATCH = 7  /* bitlinear_gemv_decode_batch_ws; N and G ignored */
 } bl_op;
 
 /* Human-readable name of a status code (static string, never NULL). */
@@ -290,6 +291,26 @@ bl_status bitlinear_gemv_decode_batch(const void* x, bl_dtype xt, int64_t M, int
                                       int b, bl_quant_mode mode, float ln_eps, int eta_correction,
                                       const uint8_t* W_packed, const float* beta, const int32_t* rowsum,
                                       void* y, bl_dtype yt, void* stream);
+
+/* bitlinear_gemv_decode_batch with a workspace (Sec. 2.1, Eq. 12, 4-7, 11 per token), for G == 1 and
+ * eta_correction == 0, M >= 2 and K <= 12288: two kernels per call.  The first quantises the tokens
+ * once (one CTA per token; LN statistics, gamma / eta, codes: the arithmetic of bitlinear_quant_act
+ * with per-token scope) into the workspace; the second streams the packed weights once per 16
+ * tokens and multiplies on the tcgen05 tensor cores (weight bit planes written to tensor memory as
+ * the A operand, int32 accumulators, exact), so the time of a call hardly depends on M up to 16.
+ * A token's result does not depend on what else is in the batch (same bits).  Other shapes, G > 1
+ * and eta_correction are handed to the kernel of bitlinear_gemv_decode_batch (workspace unused,
+ * its shape rules apply); M == 1 to that of bitlinear_gemv_decode.
+ *   x [M,K] of dtype xt;  y [M,N] of dtype yt;  W_packed in DECODE layout, read ahead of stream
+ *   order as there.  K % 256 == 0, N % 16 == 0.
+ * Workspace: BL_OP_GEMV_DECODE_BATCH (device memory, 16-byte aligned; its first word is the status
+ * word of bitlinear_ws_status: the tensor-core kernel's waits are bounded, and BL_ERR_TIMEOUT there
+ * means y of this call is not valid).  The workspace holds the codes between the two kernels, so
+ * calls that may overlap (different streams) need workspaces of their own. */
+bl_status bitlinear_gemv_decode_batch_ws(const void* x, bl_dtype xt, int64_t M, int64_t K, int64_t N, int G,
+                                         int b, bl_quant_mode mode, float ln_eps, int eta_correction,
+                                         const uint8_t* W_packed, const float* beta, const int32_t* rowsum,
+                                         void* y, bl_dtype yt, void* ws, size_t ws_bytes, void* stream);
 
 /* Causal self-attention core of the decoder block (Sec. 2, Fig. 2b; the paper keeps it in high
  * precision): per batch and head O = softmax(Q K^T / sqrt(d_h) + causal mask) V, fp16 in and out,

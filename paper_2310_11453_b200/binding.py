@@ -20,6 +20,7 @@ PER_TENSOR, PER_TOKEN = 0, 1
 CANONICAL, PREFILL, DECODE = 0, 1, 2
 OP_BINARIZE_PACK, OP_QUANT_ACT, OP_FORWARD, OP_MATMUL_I32, OP_MATMUL_DEQUANT, OP_BLOCK_FORWARD = 0, 1, 2, 3, 4, 5
 OP_FORWARD_LATENT = 6
+OP_GEMV_DECODE_BATCH = 7
 MAX_GROUPS = 64
 NOALLOC_MAX_SEGMENTS = 16384
 ERR_NULL, ERR_SHAPE, ERR_ALIGN, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_TOO_LARGE = 1, 2, 3, 4, 5, 6, 7, 8
@@ -31,6 +32,7 @@ EXPORTS = [
     "bitlinear_attention_causal", "bitlinear_block_forward", "bitlinear_ws_status",
     "bitlinear_matmul_dequant_ex", "bitlinear_binarize_pack_nsplit", "bitlinear_gemv_decode_batch",
     "bitlinear_forward_latent", "bitlinear_debug_wait_limit", "bitlinear_noalloc_status", "bitlinear_debug_decode_fallbacks",
+    "bitlinear_gemv_decode_batch_ws",
 ]
 
 _DTYPES = {torch.float32: F32, torch.float16: F16, torch.bfloat16: BF16}
@@ -92,6 +94,9 @@ def lib():
         L.bitlinear_gemv_decode_batch.restype = ci
         L.bitlinear_gemv_decode_batch.argtypes = [vp, ci, i64, i64, i64, ci, ci, ci, C.c_float, ci, vp, vp, vp, vp,
                                                   ci, vp]
+        L.bitlinear_gemv_decode_batch_ws.restype = ci
+        L.bitlinear_gemv_decode_batch_ws.argtypes = [vp, ci, i64, i64, i64, ci, ci, ci, C.c_float, ci, vp, vp, vp, vp,
+                                                     ci, vp, sz, vp]
         L.bitlinear_binarize_pack_nsplit.restype = ci
         L.bitlinear_binarize_pack_nsplit.argtypes = [vp, ci, i64, i64, ci, ci, ci, vp, vp, vp, vp, vp, vp, sz, vp]
         L.bitlinear_debug_decode_fallbacks.restype = i64
@@ -339,6 +344,21 @@ def gemv_decode_batch(x, W_packed, beta, N, G=1, mode=ABSMAX, ln_eps=1e-5, rowsu
                                              1 if eta_correction else 0, _ptr(W_packed), _ptr(beta),
                                              _ptr(rowsum), _ptr(y), _dt(y), _stream())
     _check(code, "bitlinear_gemv_decode_batch")
+    return y
+
+
+def gemv_decode_batch_ws(x, W_packed, beta, N, G=1, mode=ABSMAX, ln_eps=1e-5, rowsum=None,
+                         eta_correction=False, out_dtype=None, b=8, y=None, ws=None):
+    """bitlinear_gemv_decode_batch_ws.  x [M,K]; W_packed in DECODE layout; returns y [M,N].  `ws` may carry a
+    workspace of workspace_bytes(OP_GEMV_DECODE_BATCH, M, N, K, G) bytes (its first word is the status word)."""
+    M, K = x.shape
+    if y is None:
+        y = torch.empty((M, N), dtype=out_dtype or x.dtype, device=x.device)
+    ws = _ws(workspace_bytes(OP_GEMV_DECODE_BATCH, M, N, K, G), x.device, ws)
+    code = lib().bitlinear_gemv_decode_batch_ws(_ptr(x), _dt(x), M, K, N, G, b, mode, float(ln_eps),
+                                                1 if eta_correction else 0, _ptr(W_packed), _ptr(beta),
+                                                _ptr(rowsum), _ptr(y), _dt(y), _ptr(ws), ws.numel(), _stream())
+    _check(code, "bitlinear_gemv_decode_batch_ws")
     return y
 
 

@@ -113,6 +113,7 @@ size_t bitlinear_workspace_bytes(bl_op op, int64_t M, int64_t N, int64_t K, int 
     case BL_OP_MATMUL_DEQUANT: return (M > 0 && N > 0) ? gemm_ws_total(M, N, G) : 0;
     case BL_OP_BLOCK_FORWARD: return (M > 0 && N > 0) ? carve_block(M, K, N).total : 0;
     case BL_OP_FORWARD_LATENT: return (M > 0 && N > 0) ? carve_latent(M, N, K, G).total : 0;
+    case BL_OP_GEMV_DECODE_BATCH: return M > 0 ? round256(gemv_tc_ws_bytes(M, K)) : 0;
   }
   return 0;
 }
@@ -381,6 +382,30 @@ bl_status bitlinear_gemv_decode_batch(const void* x, bl_dtype xt, int64_t M, int
   if (!gemv_batch_supported(M, K, N, G)) return BL_ERR_SHAPE;
   if (!aligned16(x) || !aligned16(W_packed) || !aligned16(y)) return BL_ERR_ALIGN;
   GemvArgs a{x, xt, K, N, G, mode, ln_eps, eta_correction ? 1 : 0, W_packed, beta, rowsum, y, yt};
+  return launch_gemv_batch(a, M, (cudaStream_t)stream) == cudaSuccess ? BL_OK : BL_ERR_CUDA;
+}
+
+bl_status bitlinear_gemv_decode_batch_ws(const void* x, bl_dtype xt, int64_t M, int64_t K, int64_t N, int G,
+                                         int b, bl_quant_mode mode, float ln_eps, int eta_correction,
+                                         const uint8_t* W_packed, const float* beta, const int32_t* rowsum,
+                                         void* y, bl_dtype yt, void* ws, size_t ws_bytes, void* stream) {
+  if (!x || !W_packed || !beta || !y) return BL_ERR_NULL;
+  if (eta_correction && !rowsum) return BL_ERR_NULL;
+  if (M <= 0 || N <= 0) return BL_ERR_SHAPE;
+  bl_status st = check_kg(K, G);
+  if (st != BL_OK) return st;
+  if (b != 8 || !valid_dtype(xt) || !valid_dtype(yt)) return BL_ERR_UNSUPPORTED;
+  if (mode != BL_ABSMAX && mode != BL_ETA) return BL_ERR_UNSUPPORTED;
+  if (eta_correction && mode != BL_ETA) return BL_ERR_UNSUPPORTED;
+  if (!aligned16(x) || !aligned16(W_packed) || !aligned16(y)) return BL_ERR_ALIGN;
+  GemvArgs a{x, xt, K, N, G, mode, ln_eps, eta_correction ? 1 : 0, W_packed, beta, rowsum, y, yt};
+  if (gemv_tc_supported(M, K, N, G, eta_correction)) {
+    if (!ws || ws_bytes < bitlinear_workspace_bytes(BL_OP_GEMV_DECODE_BATCH, M, N, K, G)) return BL_ERR_WORKSPACE;
+    if (!aligned16(ws)) return BL_ERR_ALIGN;
+    return launch_gemv_tc(a, M, ws, (cudaStream_t)stream) == cudaSuccess ? BL_OK : BL_ERR_CUDA;
+  }
+  // shapes the tensor-core form does not take: the kernel of bitlinear_gemv_decode_batch, workspace unused
+  if (!gemv_batch_supported(M, K, N, G)) return BL_ERR_SHAPE;
   return launch_gemv_batch(a, M, (cudaStream_t)stream) == cudaSuccess ? BL_OK : BL_ERR_CUDA;
 }
 

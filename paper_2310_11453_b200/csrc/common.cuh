@@ -194,6 +194,11 @@ cudaError_t gemv_decode_take_fallbacks(unsigned int* out);   // warps that read 
 // The same for M tokens (x [M,K], y [M,N]) sharing one pass over the weights per 8 tokens.
 cudaError_t launch_gemv_batch(const GemvArgs& a, int64_t M, cudaStream_t s);
 bool gemv_batch_supported(int64_t M, int64_t K, int64_t N, int G);
+// The same with a workspace: tokens quantised once by a kernel of their own, the product on the
+// tcgen05 tensor cores, 16 tokens per pass over the weights (gemv_tc.cu).
+cudaError_t launch_gemv_tc(const GemvArgs& a, int64_t M, void* ws, cudaStream_t s);
+bool gemv_tc_supported(int64_t M, int64_t K, int64_t N, int G, int eta_correction);
+size_t gemv_tc_ws_bytes(int64_t M, int64_t K);
 
 // Decoder-block glue (fp16): the causal attention core.
 cudaError_t launch_attention_causal(const void* q, const void* k, const void* v, void* o, int batch, int S,

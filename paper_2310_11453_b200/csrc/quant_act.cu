@@ -735,6 +735,8 @@ cudaError_t run_rows(const QuantArgs& a, cudaStream_t s) {
                     (int)grid, (const ScopePartial*)partials, (const SegRecord*)recs, status, a.x_q, a.gamma, a.eta);
 }
 
+constexpr size_t kStaticSmemSlack = 4096;   // more than any kernel here declares statically
+
 template <typename T>
 cudaError_t run(const QuantArgs& a, cudaStream_t s) {
   const T* x = reinterpret_cast<const T*>(a.x);
@@ -747,7 +749,7 @@ cudaError_t run(const QuantArgs& a, cudaStream_t s) {
   if (a.gran == BL_PER_TOKEN) {
     // no device-side wait in this kernel: the word is only cleared for whoever reads it afterwards
     if (a.status && !a.keep_status && (e = cudaMemsetAsync(a.status, 0, sizeof(uint32_t), s)) != cudaSuccess) return e;
-    if (smem > 48 * 1024) {
+    if (smem + kStaticSmemSlack > 48 * 1024) {      // the 48 KB default covers static and dynamic together
       e = cudaFuncSetAttribute(quant_per_token<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e != cudaSuccess) return e;
     }
@@ -757,7 +759,7 @@ cudaError_t run(const QuantArgs& a, cudaStream_t s) {
   }
   TensorScope* sc = reinterpret_cast<TensorScope*>(reinterpret_cast<char*>(a.ws) + kWsScopeOff);
   SegRecord* recs = reinterpret_cast<SegRecord*>(reinterpret_cast<char*>(a.ws) + kWsHeaderBytes);
-  if (smem > 48 * 1024) {
+  if (smem + kStaticSmemSlack > 48 * 1024) {
     e = cudaFuncSetAttribute(tensor_stats<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }

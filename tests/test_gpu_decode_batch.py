@@ -25,6 +25,33 @@ DT = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}
     (7, 256, 32, 1, "f32", "absmax", False),         # one K block: the second warp of every pair has no work
 ])
 def test_gemv_decode_batch(M, K, N, G, dtype, mode, relu):
+    run_batch_case(B.gemv_decode_batch, M, K, N, G, dtype, mode, relu)
+
+
+# The same call with a workspace: tokens quantised by a kernel of their own, the product on the
+# tcgen05 tensor cores for G == 1 without the eta correction (other cases: the kernel above).
+@pytest.mark.parametrize("M,K,N,G,dtype,mode,relu", [
+    (8, 4096, 16384, 1, "f16", "absmax", False),     # config c2's layer, 8 tokens: 148 CTAs of 111 rows
+    (16, 4096, 16384, 1, "bf16", "absmax", False),   # a full pass of 16 tokens
+    (2, 256, 16, 1, "f32", "absmax", False),         # smallest shape: one chunk (one expander group idle), CTAs of one row
+    (3, 1024, 48, 1, "bf16", "eta", True),           # eta form without the correction
+    (37, 2048, 160, 1, "f16", "absmax", False),      # three passes, ragged last one of 5
+    (5, 8192, 20480, 1, "bf16", "absmax", False),    # 160 CTAs of 128 rows: more CTAs than SMs
+    (4, 12288, 64, 1, "f32", "absmax", False),       # the largest K: three pieces per thread of the quantiser
+    (7, 768, 3072, 1, "f32", "absmax", False),       # 125M-shaped: an odd number of chunks
+    (3, 1024, 48, 2, "bf16", "eta", True),           # groups: handed to the kernel without a workspace
+    (2, 16384, 48, 1, "f16", "absmax", False),       # K too large for the tensor-core form: likewise
+])
+def test_gemv_decode_batch_ws(M, K, N, G, dtype, mode, relu):
+    ws = torch.empty(B.workspace_bytes(B.OP_GEMV_DECODE_BATCH, M, N, K, G) + 256, dtype=torch.uint8, device=DEV)
+
+    def call(*args, **kw):
+        return B.gemv_decode_batch_ws(*args, ws=ws, **kw)
+    run_batch_case(call, M, K, N, G, dtype, mode, relu)
+    assert B.ws_status(ws) == B.OK
+
+
+def run_batch_case(gemv_decode_batch, M, K, N, G, dtype, mode, relu):
     x = synth.make_x(M, K, DT[dtype], seed=K + N + M, outliers=False, relu=relu)
     W = synth.make_w(N, K, torch.float32, seed=K)
     omode = O.ETA if mode == "eta" else O.ABSMAX
@@ -43,8 +70,8 @@ def test_gemv_decode_batch(M, K, N, G, dtype, mode, relu):
     check_codes(codes, ref_q["codes"], x=as_f32_np(x), G=G, eta_per_token=(mode == "eta"))
     acc = O.matmul(codes, w_ref["bits"], G=G)
     for corr in ([False, True] if mode == "eta" else [False]):
-        y = B.gemv_decode_batch(xd, w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode, ln_eps=1e-5,
-                                rowsum=w_gpu["rowsum"], eta_correction=corr, out_dtype=torch.float32)
+        y = gemv_decode_batch(xd, w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode, ln_eps=1e-5,
+                              rowsum=w_gpu["rowsum"], eta_correction=corr, out_dtype=torch.float32)
         torch.cuda.synchronize()
         want = O.dequant(acc, w_gpu["beta"].cpu().numpy().astype(np.float64),
                          q["gamma"].cpu().numpy().astype(np.float64), gran=O.PER_TOKEN,
@@ -61,20 +88,20 @@ def test_gemv_decode_batch(M, K, N, G, dtype, mode, relu):
         if (ties == 0).any():
             assert np.median(err[ties == 0]) <= 1e-3 * rms
     # 16-bit output is the rounding of the fp32 one
-    y32 = B.gemv_decode_batch(xd, w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode, out_dtype=torch.float32)
+    y32 = gemv_decode_batch(xd, w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode, out_dtype=torch.float32)
     if dtype != "f32":
-        y16 = B.gemv_decode_batch(xd, w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode, out_dtype=DT[dtype])
+        y16 = gemv_decode_batch(xd, w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode, out_dtype=DT[dtype])
         assert torch.equal(y16, y32.to(DT[dtype]))
     # a token's result does not depend on what else is in the batch: the last two tokens as a batch of
     # their own give the same bits (a single token takes the single-token kernel, whose sums run in
     # another order: same codes up to the tolerated ties, gamma to the last bit or so)
     if M > 2:
-        y_two = B.gemv_decode_batch(xd[M - 2:M].contiguous(), w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode,
-                                    out_dtype=torch.float32)
+        y_two = gemv_decode_batch(xd[M - 2:M].contiguous(), w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode,
+                                  out_dtype=torch.float32)
         assert torch.equal(y_two, y32[M - 2:M])
     if M > 1:
-        y_one = B.gemv_decode_batch(xd[M - 1:M].contiguous(), w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode,
-                                    out_dtype=torch.float32)
+        y_one = gemv_decode_batch(xd[M - 1:M].contiguous(), w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode,
+                                  out_dtype=torch.float32)
         d = np.abs(y_one[0].cpu().numpy().astype(np.float64) - y32[M - 1].cpu().numpy().astype(np.float64))
         assert (d <= 1e-3 * rms + slack[M - 1]).all()
 

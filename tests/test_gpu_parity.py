@@ -182,6 +182,8 @@ QUANT_CASES = [
     (40, 8192, 1, "f16", "eta", "token", False, True),       # more 16 KB segments than warps in a CTA
     (5, 16384, 1, "bf16", "absmax", "token", True, False),   # longer than a warp's staging area: CTA path
     (5, 16384, 1, "bf16", "eta", "tensor", False, True),
+    (4, 12288, 1, "f32", "absmax", "token", False, False),   # CTA path with exactly 48 KB of dynamic shared memory
+    (4, 12288, 1, "f32", "eta", "tensor", False, True),
     # per-tensor scope in one kernel: segments per CTA below, at and above what stays in shared memory
     (1, 4096, 1, "bf16", "absmax", "tensor", False, False),
     (3600, 512, 1, "bf16", "eta", "tensor", False, True),    # 24-25 segments per CTA
