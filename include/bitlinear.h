@@ -293,14 +293,16 @@ bl_status bitlinear_gemv_decode_batch(const void* x, bl_dtype xt, int64_t M, int
                                       void* y, bl_dtype yt, void* stream);
 
 /* bitlinear_gemv_decode_batch with a workspace (Sec. 2.1, Eq. 12, 4-7, 11 per token), for G == 1 and
- * eta_correction == 0, M >= 2 and K <= 12288: two kernels per call.  The first quantises the tokens
+ * eta_correction == 0, M >= 8 and K <= 12288: two kernels per call.  The first quantises the tokens
  * once (one CTA per token; LN statistics, gamma / eta, codes: the arithmetic of bitlinear_quant_act
  * with per-token scope) into the workspace; the second streams the packed weights once per 16
  * tokens and multiplies on the tcgen05 tensor cores (weight bit planes written to tensor memory as
  * the A operand, int32 accumulators, exact), so the time of a call hardly depends on M up to 16.
- * A token's result does not depend on what else is in the batch (same bits).  Other shapes, G > 1
- * and eta_correction are handed to the kernel of bitlinear_gemv_decode_batch (workspace unused,
- * its shape rules apply); M == 1 to that of bitlinear_gemv_decode.
+ * A token's result does not depend on what else is in the batch as long as the batch stays on the
+ * same side of 8 tokens (same bits).  Fewer than 8 tokens, other shapes, G > 1 and eta_correction
+ * are handed to the kernel of bitlinear_gemv_decode_batch where it takes the shape (workspace
+ * unused, its shape rules apply; for fewer than 8 tokens it is as fast or faster); M == 1 to that
+ * of bitlinear_gemv_decode.
  *   x [M,K] of dtype xt;  y [M,N] of dtype yt;  W_packed in DECODE layout, read ahead of stream
  *   order as there.  K % 256 == 0, N % 16 == 0.
  * Workspace: BL_OP_GEMV_DECODE_BATCH (device memory, 16-byte aligned; its first word is the status

@@ -33,25 +33,27 @@ def test_gemv_decode_batch(M, K, N, G, dtype, mode, relu):
 @pytest.mark.parametrize("M,K,N,G,dtype,mode,relu", [
     (8, 4096, 16384, 1, "f16", "absmax", False),     # config c2's layer, 8 tokens: 148 CTAs of 111 rows
     (16, 4096, 16384, 1, "bf16", "absmax", False),   # a full pass of 16 tokens
-    (2, 256, 16, 1, "f32", "absmax", False),         # smallest shape: one chunk (one expander group idle), CTAs of one row
-    (3, 1024, 48, 1, "bf16", "eta", True),           # eta form without the correction
+    (8, 256, 16, 1, "f32", "absmax", False),         # smallest shape: one chunk (half a slot), CTAs of one row
+    (9, 1024, 48, 1, "bf16", "eta", True),           # eta form without the correction; the second half of the codes is used
     (37, 2048, 160, 1, "f16", "absmax", False),      # three passes, ragged last one of 5
-    (5, 8192, 20480, 1, "bf16", "absmax", False),    # 160 CTAs of 128 rows: more CTAs than SMs
-    (4, 12288, 64, 1, "f32", "absmax", False),       # the largest K: three pieces per thread of the quantiser
-    (7, 768, 3072, 1, "f32", "absmax", False),       # 125M-shaped: an odd number of chunks
-    (3, 1024, 48, 2, "bf16", "eta", True),           # groups: handed to the kernel without a workspace
-    (2, 16384, 48, 1, "f16", "absmax", False),       # K too large for the tensor-core form: likewise
+    (11, 8192, 20480, 1, "bf16", "absmax", False),   # 160 CTAs of 128 rows: more CTAs than SMs
+    (8, 12288, 64, 1, "f32", "absmax", False),       # the largest K: six pieces per thread of the quantiser
+    (10, 768, 3072, 1, "f32", "absmax", False),      # 125M-shaped: an odd number of chunks
+    (4, 4096, 1024, 1, "f16", "absmax", False),      # fewer than 8 tokens: the kernel without a workspace
+    (9, 1024, 48, 2, "bf16", "eta", True),           # groups: likewise
+    (8, 16384, 48, 1, "f16", "absmax", False),       # K too large for the tensor-core form: likewise
 ])
 def test_gemv_decode_batch_ws(M, K, N, G, dtype, mode, relu):
     ws = torch.empty(B.workspace_bytes(B.OP_GEMV_DECODE_BATCH, M, N, K, G) + 256, dtype=torch.uint8, device=DEV)
 
     def call(*args, **kw):
         return B.gemv_decode_batch_ws(*args, ws=ws, **kw)
-    run_batch_case(call, M, K, N, G, dtype, mode, relu)
+    # below 8 tokens the call runs another kernel: same bits are promised among batches of 8 or more
+    run_batch_case(call, M, K, N, G, dtype, mode, relu, same_bits_from=8 if (G == 1 and K <= 12288) else 2)
     assert B.ws_status(ws) == B.OK
 
 
-def run_batch_case(gemv_decode_batch, M, K, N, G, dtype, mode, relu):
+def run_batch_case(gemv_decode_batch, M, K, N, G, dtype, mode, relu, same_bits_from=2):
     x = synth.make_x(M, K, DT[dtype], seed=K + N + M, outliers=False, relu=relu)
     W = synth.make_w(N, K, torch.float32, seed=K)
     omode = O.ETA if mode == "eta" else O.ABSMAX
@@ -92,13 +94,14 @@ def run_batch_case(gemv_decode_batch, M, K, N, G, dtype, mode, relu):
     if dtype != "f32":
         y16 = gemv_decode_batch(xd, w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode, out_dtype=DT[dtype])
         assert torch.equal(y16, y32.to(DT[dtype]))
-    # a token's result does not depend on what else is in the batch: the last two tokens as a batch of
+    # a token's result does not depend on what else is in the batch: the last tokens as a (smallest) batch of
     # their own give the same bits (a single token takes the single-token kernel, whose sums run in
     # another order: same codes up to the tolerated ties, gamma to the last bit or so)
-    if M > 2:
-        y_two = gemv_decode_batch(xd[M - 2:M].contiguous(), w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode,
+    if M > same_bits_from:
+        sub = same_bits_from
+        y_sub = gemv_decode_batch(xd[M - sub:M].contiguous(), w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode,
                                   out_dtype=torch.float32)
-        assert torch.equal(y_two, y32[M - 2:M])
+        assert torch.equal(y_sub, y32[M - sub:M])
     if M > 1:
         y_one = gemv_decode_batch(xd[M - 1:M].contiguous(), w_gpu["W_packed"], w_gpu["beta"], N, G=G, mode=omode,
                                   out_dtype=torch.float32)
