@@ -294,10 +294,11 @@ bl_status bitlinear_gemv_decode_batch(const void* x, bl_dtype xt, int64_t M, int
 
 /* bitlinear_gemv_decode_batch with a workspace (Sec. 2.1, Eq. 12, 4-7, 11 per token), for G == 1 and
  * eta_correction == 0, M >= 8 and K <= 12288: two kernels per call.  The first quantises the tokens
- * once (one CTA per token; LN statistics, gamma / eta, codes: the arithmetic of bitlinear_quant_act
- * with per-token scope) into the workspace; the second streams the packed weights once per 16
- * tokens and multiplies on the tcgen05 tensor cores (weight bit planes written to tensor memory as
- * the A operand, int32 accumulators, exact), so the time of a call hardly depends on M up to 16.
+ * once (one CTA per token; LN statistics, gamma / eta, codes: the fp32 arithmetic of the kernel
+ * of bitlinear_gemv_decode) into the workspace; the second streams the packed weights once per 32
+ * tokens (per 16 when K > 6144) and multiplies on the tcgen05 tensor cores (weight bit planes
+ * written to tensor memory as the A operand, int32 accumulators, exact), so the time of a call
+ * depends little on M up to 32.
  * A token's result does not depend on what else is in the batch as long as the batch stays on the
  * same side of 8 tokens (same bits).  Fewer than 8 tokens, other shapes, G > 1 and eta_correction
  * are handed to the kernel of bitlinear_gemv_decode_batch where it takes the shape (workspace

@@ -12,7 +12,7 @@
 //
 //   gemv_tc_kernel        the product, transposed: y^T = W~ x~^T.  A CTA owns up to 128 weight
 //                         rows (the M side of tcgen05.mma kind::i8, 128 x 16 x 32) and all of K;
-//                         up to 16 tokens are the 16 columns.  The weights never pass through
+//                         up to 16 (or 32) tokens are the columns.  The weights never pass through
 //                         shared memory: a thread owns one row (= one lane of tensor memory),
 //                         reads 256 of its weights (32 bytes) from global memory / L2, and for
 //                         bit plane j forms word & (0x01010101 << j) - in DECODE layout that is
@@ -23,7 +23,7 @@
 //                         sums 2^j (-128 for j = 7) times the codes under its set bits; the
 //                         epilogue adds acc_j >> j over the planes (exact) and applies
 //                         sum_k W~ x~ = 2 sum_{bit=1} x~ - sum x~ and the Eq. 11 rescale.
-//                         The B operand (16 tokens x 32 codes per MMA) comes from shared memory,
+//                         The B operand (the tokens x 32 codes per MMA) comes from shared memory,
 //                         copied there in one piece from the workspace.
 //
 // Issue rate.  One thread issues a tcgen05.mma in about 63 clocks and a commit in about 67
@@ -49,20 +49,20 @@ namespace {
 
 using namespace tc;
 
-constexpr int kTok = 16;                 // tokens per pass (MMA N)
+constexpr int kTokMax = 32;              // tokens per pass (MMA N): 16, or 32 where their codes fit in shared memory
 constexpr int kQuantThreads = 256;        // with the product kernel's 384 threads on the same SM: registers for both
 constexpr int kQuantWarps = kQuantThreads / 32;
 constexpr int kMaxOctets = 6;            // 8-feature pieces per thread of the quantising kernel: K <= 12288
 constexpr int kTcThreads = 384;          // warps 0-7 expand (0-3 also run the epilogue), 8-11 issue
-constexpr int kSlots = 3;                // A ring: slots per expander group, two chunks (four planes of each) per slot
+constexpr int kSlotsMax = 3;             // A ring: slots per expander group (3 for 16 tokens, 2 for 32), two chunks x four planes per slot
 constexpr int kSlotCols = 64;            // 2 chunks x 4 planes x 8 columns (32 bytes of K per lane and plane)
-constexpr uint32_t kColA = 128;          // accumulators: columns 0..127 = [plane 8][token 16]; A ring [group 2][slot 3] behind
+                                         // accumulators: columns [plane 8][token NT]; the A ring [group 2][slot] behind them
 constexpr uint32_t kTmemCols = 512;
 constexpr size_t kStatusBytes = 256;
-constexpr size_t kTailBytes = 128;       // gamma[16] (float), csum[16] (int) behind the codes of a pass
 constexpr uint32_t kCopyPiece = 16384;
 
-__host__ __device__ inline size_t pass_bytes(int64_t K) { return (size_t)kTok * (size_t)K + kTailBytes; }
+// a pass: the codes of nt tokens, then gamma[nt] (float) and csum[nt] (int)
+__host__ __device__ inline size_t pass_bytes(int64_t K, int nt) { return (size_t)nt * ((size_t)K + 8); }
 
 // Where the code of feature k of token n sits in a pass's code block.  The block is B tiles of 8
 // token rows x 128 bytes, [token half n / 8][tile K / 128][row n % 8][128 bytes], 128-byte swizzled
@@ -80,6 +80,7 @@ __device__ __forceinline__ uint32_t code_offset4(int k, int n, int tiles) {   //
 struct QuantTokArgs {
   const void* x; int64_t K; int mode; float ln_eps;
   float inv_k; double inv_k_d;
+  int nt;                   // tokens per pass
   uint8_t* passes;          // workspace behind the status block
   uint32_t* status;         // cleared here (in stream order); the product kernels only ever raise it
 };
@@ -114,8 +115,8 @@ __global__ void __launch_bounds__(kQuantThreads, 2) decode_quant_kernel(QuantTok
   __shared__ int red_c[kQuantWarps];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t m = blockIdx.x;
-  const int n = (int)(m % kTok);
-  uint8_t* region = a.passes + (size_t)(m / kTok) * pass_bytes(a.K);
+  const int n = (int)(m % a.nt);
+  uint8_t* region = a.passes + (size_t)(m / a.nt) * pass_bytes(a.K, a.nt);
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");     // the product kernel may start on the weights
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (m == 0 && threadIdx.x == 0) *a.status = 0u;
@@ -193,7 +194,7 @@ __global__ void __launch_bounds__(kQuantThreads, 2) decode_quant_kernel(QuantTok
         rstd = rstd_outside_fp32(vv);
       }
     }
-    reinterpret_cast<float*>(region + (size_t)kTok * (size_t)a.K)[n] = span_f * rstd;
+    reinterpret_cast<float*>(region + (size_t)a.nt * (size_t)a.K)[n] = span_f * rstd;
   }
   // ---- Eq. 4 / 6: codes, written where the product kernel's MMAs read them ---------------------------
   int csum = 0;
@@ -238,21 +239,21 @@ __global__ void __launch_bounds__(kQuantThreads, 2) decode_quant_kernel(QuantTok
     int t = red_c[threadIdx.x];
 #pragma unroll
     for (int o = kQuantWarps / 2; o > 0; o >>= 1) t += __shfl_xor_sync((1u << kQuantWarps) - 1u, t, o);
-    if (threadIdx.x == 0) reinterpret_cast<int*>(region + (size_t)kTok * (size_t)a.K)[kTok + n] = t;
+    if (threadIdx.x == 0) reinterpret_cast<int*>(region + (size_t)a.nt * (size_t)a.K)[a.nt + n] = t;
   }
 }
 
 // ---- the product ------------------------------------------------------------------------------------
 struct TcArgs {
   const uint8_t* W; int64_t K, N; int rows_per_cta;
-  const uint8_t* region;     // codes of this pass | gamma[16] | csum[16]
+  const uint8_t* region;     // codes of this pass | gamma[NT] | csum[NT]
   const float* beta;
   void* y; int64_t m0; int mcount;
   uint32_t* status;
 };
 
 struct TcShared {
-  unsigned long long full[2][kSlots], empty[2][kSlots], codes_full, acc_full;
+  unsigned long long full[2][kSlotsMax], empty[2][kSlotsMax], codes_full, acc_full;
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -290,11 +291,13 @@ __device__ __forceinline__ uint64_t smem_desc_sw128_sbo(uint32_t addr, uint32_t 
   return d;
 }
 
-// kind::i8 instruction descriptor: s32 accumulate, s8 x s8, both operands K-major, 128 x 16.
-constexpr uint32_t kIdesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTok >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-
-template <typename TY>
+// NT: tokens per pass, 16 or 32.
+template <typename TY, int NT>
 __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(TcArgs a) {
+  // kind::i8 instruction descriptor: s32 accumulate, s8 x s8, both operands K-major, 128 x NT.
+  constexpr uint32_t kIdesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+  constexpr uint32_t kColA = 8u * NT;
+  constexpr int kSlots = (int)((kTmemCols - kColA) / (2 * kSlotCols));
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* codes = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   __shared__ TcShared sh;
@@ -305,7 +308,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(TcArgs a) {
   const int npairs = (nchunks + 1) >> 1;
   const int64_t row_begin = (int64_t)blockIdx.x * a.rows_per_cta;
   const int rows_cta = (int)min((int64_t)a.rows_per_cta, a.N - row_begin);
-  const uint32_t half_bytes = 8u * (uint32_t)a.K;          // the codes of 8 tokens: all tiles of rows 0..7, then of rows 8..15
+  const uint32_t half_bytes = 8u * (uint32_t)a.K;          // the codes of 8 tokens: all tiles of rows 0..7, then of rows 8..15, ...
 
   if (threadIdx.x == 0) {
     for (int g = 0; g < 2; ++g)
@@ -391,7 +394,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(TcArgs a) {
   } else if (lane == 0) {
     // ------------------------------------------------------------------ issuers: two planes each, every chunk
     const int i = warp - 8, g = i >> 1, j0 = 4 * g + 2 * (i & 1);
-    const uint32_t copy_bytes = a.mcount > 8 ? 2u * half_bytes : half_bytes;
+    const uint32_t copy_bytes = (uint32_t)((a.mcount + 7) >> 3) * half_bytes;
     if (i == 0) {
       asm volatile("griddepcontrol.wait;" ::: "memory");              // the codes are the work of the kernel before
       mbar_arrive_expect_tx(smem_u32(&sh.codes_full), copy_bytes);
@@ -418,7 +421,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(TcArgs a) {
 #pragma unroll
           for (int t = 0; t < 2; ++t) {
             const int j = j0 + t;
-            mma_i8_ts(tmem_base + (uint32_t)(j * kTok), abase + (uint32_t)(cc * 32 + (j & 3) * 8),
+            mma_i8_ts(tmem_base + (uint32_t)(j * NT), abase + (uint32_t)(cc * 32 + (j & 3) * 8),
                       bdesc + (uint64_t)(2 * (j & 3)), kIdesc, c > 0 ? 1u : 0u);
           }
         }
@@ -434,38 +437,42 @@ __global__ void __launch_bounds__(kTcThreads, 1) gemv_tc_kernel(TcArgs a) {
     // ------------------------------------------------------------------ epilogue: thread = weight row
     asm volatile("griddepcontrol.wait;" ::: "memory");                // gamma, csum; y in stream order
     // lane n holds what token n needs (fetched while the last MMAs run)
-    const float* tail = reinterpret_cast<const float*>(a.region + 2u * half_bytes);
-    const float my_scale = __ldg(a.beta) * tail[lane & (kTok - 1)] * kInvQb;
-    const int my_csum = reinterpret_cast<const int*>(tail)[kTok + (lane & (kTok - 1))];
+    const float* tail = reinterpret_cast<const float*>(a.region + (uint32_t)NT * (uint32_t)a.K);
+    const float my_scale = __ldg(a.beta) * tail[lane & (NT - 1)] * kInvQb;
+    const int my_csum = reinterpret_cast<const int*>(tail)[NT + (lane & (NT - 1))];
     bool ok = true;
     if (lane == 0) ok = mbar_wait(smem_u32(&sh.acc_full), 0u, abort_flag);
     ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
     tc_fence_after();
     if (ok) {
       const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-      int S[kTok];
-#pragma unroll
-      for (int n = 0; n < kTok; ++n) S[n] = 0;
-#pragma unroll
-      for (int jb = 0; jb < 8; jb += 4) {
-        uint32_t d[4][kTok];
-#pragma unroll
-        for (int t = 0; t < 4; ++t) tmem_ld16_nowait(tmem_base + lane_base + (uint32_t)((jb + t) * kTok), d[t]);
-        tmem_ld_wait();
-        // plane j holds 2^j * (sum of the codes under its set bits); the byte 0x80 of plane 7 is -128
-#pragma unroll
-        for (int t = 0; t < 4; ++t)
-#pragma unroll
-          for (int n = 0; n < kTok; ++n) S[n] += (jb + t < 7) ? ((int)d[t][n] >> (jb + t)) : -((int)d[t][n] >> 7);
-      }
       const int row = warp * 32 + lane;
       TY* y = reinterpret_cast<TY*>(a.y);
+#pragma unroll 1
+      for (int n0 = 0; n0 < NT && n0 < a.mcount; n0 += 16) {         // 16 tokens (accumulator columns) at a time
+        int S[16];
 #pragma unroll
-      for (int n = 0; n < kTok; ++n) {
-        const float sc = __shfl_sync(0xFFFFFFFFu, my_scale, n);
-        const int cs = __shfl_sync(0xFFFFFFFFu, my_csum, n);
-        // Eq. 7 and 11: (2 S - sum x~) beta gamma / Q_b
-        if (n < a.mcount && row < rows_cta) y[(a.m0 + n) * a.N + row_begin + row] = out_cast<TY>((float)(2 * S[n] - cs) * sc);
+        for (int n = 0; n < 16; ++n) S[n] = 0;
+#pragma unroll
+        for (int jb = 0; jb < 8; jb += 4) {
+          uint32_t d[4][16];
+#pragma unroll
+          for (int t = 0; t < 4; ++t) tmem_ld16_nowait(tmem_base + lane_base + (uint32_t)((jb + t) * NT + n0), d[t]);
+          tmem_ld_wait();
+          // plane j holds 2^j * (sum of the codes under its set bits); the byte 0x80 of plane 7 is -128
+#pragma unroll
+          for (int t = 0; t < 4; ++t)
+#pragma unroll
+            for (int n = 0; n < 16; ++n) S[n] += (jb + t < 7) ? ((int)d[t][n] >> (jb + t)) : -((int)d[t][n] >> 7);
+        }
+#pragma unroll
+        for (int n = 0; n < 16; ++n) {
+          const float sc = __shfl_sync(0xFFFFFFFFu, my_scale, n0 + n);
+          const int cs = __shfl_sync(0xFFFFFFFFu, my_csum, n0 + n);
+          // Eq. 7 and 11: (2 S - sum x~) beta gamma / Q_b
+          if (n0 + n < a.mcount && row < rows_cta)
+            y[(a.m0 + n0 + n) * a.N + row_begin + row] = out_cast<TY>((float)(2 * S[n] - cs) * sc);
+        }
       }
     }
   }
@@ -511,15 +518,18 @@ cudaError_t run(const GemvArgs& a, int64_t M, void* ws, cudaStream_t s) {
   // second one on the same SM (the next call's, or one displaced from an SM that is full) would sit in
   // tcgen05.alloc behind it and then start with an empty ring.  Asking for more than half of the
   // shared memory keeps them apart; a waiting CTA then takes the first SM that frees up.
-  const size_t smem = std::max<size_t>((size_t)kTok * (size_t)a.K + 1024, 116 * 1024);
+  const int nt = (M > 16 && (size_t)32 * (size_t)a.K + 1024 <= 200 * 1024) ? 32 : 16;
+  const size_t smem = std::max<size_t>((size_t)nt * (size_t)a.K + 1024, 116 * 1024);
   static std::atomic<int> configured[64];
   if (dev >= 64 || !configured[dev].load(std::memory_order_acquire)) {
-    e = cudaFuncSetAttribute(gemv_tc_kernel<TY>, cudaFuncAttributeMaxDynamicSharedMemorySize, 216 * 1024);
+    e = cudaFuncSetAttribute(gemv_tc_kernel<TY, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 216 * 1024);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(gemv_tc_kernel<TY, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, 216 * 1024);
     if (e != cudaSuccess) return e;
     if (dev < 64) configured[dev].store(1, std::memory_order_release);
   }
   uint8_t* base = reinterpret_cast<uint8_t*>(ws);
-  QuantTokArgs qa{a.x, a.K, (int)a.mode, a.ln_eps, (float)(1.0 / (double)a.K), 1.0 / (double)a.K, base + kStatusBytes,
+  QuantTokArgs qa{a.x, a.K, (int)a.mode, a.ln_eps, (float)(1.0 / (double)a.K), 1.0 / (double)a.K, nt, base + kStatusBytes,
                   reinterpret_cast<uint32_t*>(base)};
   const int64_t per_thread = (a.K / 8 + kQuantThreads - 1) / kQuantThreads;
   if (per_thread <= 2) e = launch_pdl(decode_quant_kernel<TX, 2>, dim3((unsigned)M), dim3(kQuantThreads), 0, s, qa);
@@ -528,10 +538,11 @@ cudaError_t run(const GemvArgs& a, int64_t M, void* ws, cudaStream_t s) {
   if (e != cudaSuccess) return e;
   const int rows_per_cta = (int)std::min<int64_t>(128, (a.N + sms - 1) / sms);
   const unsigned grid = (unsigned)((a.N + rows_per_cta - 1) / rows_per_cta);
-  for (int64_t m0 = 0; m0 < M; m0 += kTok) {
-    TcArgs ta{a.W_packed, a.K, a.N, rows_per_cta, base + kStatusBytes + (size_t)(m0 / kTok) * pass_bytes(a.K), a.beta,
-              a.y, m0, (int)std::min<int64_t>(kTok, M - m0), reinterpret_cast<uint32_t*>(base)};
-    e = launch_pdl(gemv_tc_kernel<TY>, dim3(grid), dim3(kTcThreads), smem, s, ta);
+  for (int64_t m0 = 0; m0 < M; m0 += nt) {
+    TcArgs ta{a.W_packed, a.K, a.N, rows_per_cta, base + kStatusBytes + (size_t)(m0 / nt) * pass_bytes(a.K, nt), a.beta,
+              a.y, m0, (int)std::min<int64_t>(nt, M - m0), reinterpret_cast<uint32_t*>(base)};
+    e = nt == 32 ? launch_pdl(gemv_tc_kernel<TY, 32>, dim3(grid), dim3(kTcThreads), smem, s, ta)
+                 : launch_pdl(gemv_tc_kernel<TY, 16>, dim3(grid), dim3(kTcThreads), smem, s, ta);
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;
@@ -555,7 +566,7 @@ bool gemv_tc_supported(int64_t M, int64_t K, int64_t N, int G, int eta_correctio
 }
 
 size_t gemv_tc_ws_bytes(int64_t M, int64_t K) {
-  return kStatusBytes + (size_t)((M + kTok - 1) / kTok) * pass_bytes(K);
+  return kStatusBytes + (size_t)((M + 31) / 32) * pass_bytes(K, 32);      // covers passes of 16 as well
 }
 
 cudaError_t launch_gemv_tc(const GemvArgs& a, int64_t M, void* ws, cudaStream_t s) {

@@ -35,7 +35,10 @@ def test_gemv_decode_batch(M, K, N, G, dtype, mode, relu):
     (16, 4096, 16384, 1, "bf16", "absmax", False),   # a full pass of 16 tokens
     (8, 256, 16, 1, "f32", "absmax", False),         # smallest shape: one chunk (half a slot), CTAs of one row
     (9, 1024, 48, 1, "bf16", "eta", True),           # eta form without the correction; the second half of the codes is used
-    (37, 2048, 160, 1, "f16", "absmax", False),      # three passes, ragged last one of 5
+    (37, 2048, 160, 1, "f16", "absmax", False),      # passes of 32 tokens: a full one and a ragged one of 5
+    (32, 4096, 16384, 1, "f16", "absmax", False),    # one pass of 32 tokens at config c2's layer
+    (17, 6144, 256, 1, "bf16", "eta", True),         # the largest K with 32 tokens per pass; 17 tokens: three of four token blocks
+    (20, 8192, 64, 1, "f16", "absmax", False),       # more than 16 tokens with K too large for 32 per pass: two passes of 16
     (11, 8192, 20480, 1, "bf16", "absmax", False),   # 160 CTAs of 128 rows: more CTAs than SMs
     (8, 12288, 64, 1, "f32", "absmax", False),       # the largest K: six pieces per thread of the quantiser
     (10, 768, 3072, 1, "f32", "absmax", False),      # 125M-shaped: an odd number of chunks
