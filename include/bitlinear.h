@@ -301,9 +301,9 @@ bl_status bitlinear_gemv_decode_batch(const void* x, bl_dtype xt, int64_t M, int
  * depends little on M up to 32.
  * A token's result does not depend on what else is in the batch as long as the batch stays on the
  * same side of 8 tokens (same bits).  Fewer than 8 tokens, other shapes, G > 1 and eta_correction
- * are handed to the kernel of bitlinear_gemv_decode_batch where it takes the shape (workspace
- * unused, its shape rules apply; for fewer than 8 tokens it is as fast or faster); M == 1 to that
- * of bitlinear_gemv_decode.
+ * are handed to the kernel of bitlinear_gemv_decode_batch where it takes the shape (of the
+ * workspace only the status word is used: cleared; its shape rules apply; for fewer than 8 tokens
+ * it is as fast or faster); M == 1 to that of bitlinear_gemv_decode.
  *   x [M,K] of dtype xt;  y [M,N] of dtype yt;  W_packed in DECODE layout, read ahead of stream
  *   order as there.  K % 256 == 0, N % 16 == 0.
  * Workspace: BL_OP_GEMV_DECODE_BATCH (device memory, 16-byte aligned; its first word is the status

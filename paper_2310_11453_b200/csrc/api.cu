@@ -407,7 +407,9 @@ bl_status bitlinear_gemv_decode_batch_ws(const void* x, bl_dtype xt, int64_t M, 
     if (!aligned16(ws)) return BL_ERR_ALIGN;
     return launch_gemv_tc(a, M, ws, (cudaStream_t)stream) == cudaSuccess ? BL_OK : BL_ERR_CUDA;
   }
-  // shapes the tensor-core form does not take: the kernel of bitlinear_gemv_decode_batch, workspace unused
+  // shapes the tensor-core form does not take: the kernel of bitlinear_gemv_decode_batch; of the workspace
+  // only the status word is touched (cleared, so that bitlinear_ws_status answers for this call too)
+  if (ws && ws_bytes >= sizeof(uint32_t) && aligned16(ws)) a.clear_status = reinterpret_cast<uint32_t*>(ws);
   if (!gemv_batch_supported(M, K, N, G)) return BL_ERR_SHAPE;
   return launch_gemv_batch(a, M, (cudaStream_t)stream) == cudaSuccess ? BL_OK : BL_ERR_CUDA;
 }

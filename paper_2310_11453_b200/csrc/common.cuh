@@ -188,6 +188,7 @@ struct GemvArgs {
   const void* x; bl_dtype xt; int64_t K, N; int G; bl_quant_mode mode; float ln_eps;
   int eta_correction; const uint8_t* W_packed; const float* beta; const int32_t* rowsum;
   void* y; bl_dtype yt;
+  uint32_t* clear_status = nullptr;   // when set: a status word that the call's (first) kernel clears, in stream order
 };
 cudaError_t launch_gemv_decode(const GemvArgs& a, cudaStream_t s);
 cudaError_t gemv_decode_take_fallbacks(unsigned int* out);   // warps that read weights from global memory after a wait ran out

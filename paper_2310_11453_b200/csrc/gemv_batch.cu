@@ -72,6 +72,7 @@ struct BatchArgs {
   const uint8_t* W_packed; const float* beta; const int32_t* rowsum; void* y;
   int stage_tokens;                      // the raw tokens fit in shared memory beside the codes
   double inv_kg;                         // 1 / K_g (a double-precision division per thread otherwise)
+  uint32_t* clear_status;                // when set: a status word this launch clears, in stream order
 };
 
 // The four A words of K block b for this lane: rows g and g + 8, words qd and 4 + qd of the block.
@@ -132,6 +133,7 @@ gemv_batch_kernel(BatchArgs a) {
   if (threadIdx.x < kZeroBytes / 4) reinterpret_cast<uint32_t*>(smem)[threadIdx.x] = 0u;
   pdl_launch_dependents();
   pdl_wait();
+  if (a.clear_status != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *a.clear_status = 0u;
 
   // ---- 2. LN + Quant of the tokens
   if (a.stage_tokens) {
@@ -398,6 +400,7 @@ cudaError_t launch_gemv_batch(const GemvArgs& g, int64_t M, cudaStream_t s) {
     a.y = reinterpret_cast<char*>(g.y) + (size_t)m0 * (size_t)g.N * ysz;
     a.stage_tokens = 0;
     a.inv_kg = 1.0 / (double)(g.K / g.G);
+    a.clear_status = m0 == 0 ? g.clear_status : nullptr;
     cudaError_t e = cudaErrorInvalidValue;
     switch (g.xt) {
       case BL_F32: e = run1<float>(a, g.yt, s); break;

@@ -540,6 +540,7 @@ gemv_decode_kernel(GemvArgs a, GemvGeom geo) {
   __syncthreads();
   BL_STAMP(11);
   BL_STAMP_NS(2);
+  if (threadIdx.x == 0 && blockIdx.x == 0 && a.clear_status != nullptr) *a.clear_status = 0u;
   if (threadIdx.x == 0 && sh.abandon) {
     const unsigned long long t0 = global_ns();
     for (int slot = 0; slot < depth; ++slot) {
@@ -934,6 +935,7 @@ gemv_decode_fast_kernel(GemvArgs a, FastGeom geo) {
   __syncthreads();
   BL_STAMP(13);
   BL_STAMP_NS(2);
+  if (threadIdx.x == 0 && blockIdx.x == 0 && a.clear_status != nullptr) *a.clear_status = 0u;
   if (threadIdx.x == 0 && sh.abandon) {
     const unsigned long long t0 = global_ns();
     for (int slot = 0; slot < depth; ++slot) {

@@ -72,3 +72,24 @@ def test_random_shapes_against_the_oracle(seed):
         except B.BitLinearError as e:
             assert e.code in (B.ERR_SHAPE, B.ERR_UNSUPPORTED), e   # outside the documented limits: refused, not wrong
     assert ran >= DRAWS_PER_SEED // 2
+
+
+@pytest.mark.parametrize("seed", [21, 22])
+def test_random_shapes_decode_batch_with_a_workspace(seed):
+    # The tensor-core form (8 or more tokens, one group, K up to 12288) and the hand-over to the other
+    # decode kernels around it: token counts on both sides of 8, 16 and 32, chunk counts odd and even,
+    # K on both sides of the 32-tokens-per-pass limit, row counts that leave the last CTA short.
+    rng = random.Random(seed)
+    ran = 0
+    for _ in range(30):
+        G = rng.choice([1, 1, 1, 1, 2])
+        M = rng.choice([2, 7, 8, 9, 15, 16, 17, 24, 31, 32, 33, 40])
+        K = 256 * G * rng.randint(1, 48 // G)
+        N = 16 * rng.choice([1, 2, 7, 9, 10, 37, 148, 149, 300])
+        dtype, mode = rng.choice(["f32", "f16", "bf16"]), rng.choice(["absmax", "eta"])
+        try:
+            TB.test_gemv_decode_batch_ws(M, K, N, G, dtype, mode, mode == "eta" and rng.random() < 0.7)
+            ran += 1
+        except B.BitLinearError as e:
+            assert e.code in (B.ERR_SHAPE, B.ERR_UNSUPPORTED), e
+    assert ran >= 20
