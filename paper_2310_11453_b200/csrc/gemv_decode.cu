@@ -570,6 +570,7 @@ struct FastGeom {            // decided on the host
   uint32_t stage_stride;     // bytes between ring slots (a multiple of 128)
   uint32_t ring_bytes;       // depth * stage_stride
   uint32_t wait_polls;
+  int x_in_smem;             // more than one slice and not kept in registers: raw x as fp32 in shared memory
   float inv_k;
   double inv_k_d;
 };
@@ -618,6 +619,22 @@ __device__ __forceinline__ void warp_rows(const uint32_t (&xr)[32], int rpw, uin
   }
 }
 
+// Eight 16-bit inputs (one 16-byte load) as floats.
+template <typename T> __device__ __forceinline__ void unpack8(const uint4& r, float (&v)[8]);
+template <> __device__ __forceinline__ void unpack8<__half>(const uint4& r, float (&v)[8]) {
+  const __half2* h = reinterpret_cast<const __half2*>(&r);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { const float2 f = __half22float2(h[i]); v[2 * i] = f.x; v[2 * i + 1] = f.y; }
+}
+template <> __device__ __forceinline__ void unpack8<__nv_bfloat16>(const uint4& r, float (&v)[8]) {
+  const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { v[2 * i] = __uint_as_float(w[i] << 16); v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u); }
+}
+template <> __device__ __forceinline__ void unpack8<float>(const uint4&, float (&)[8]) {}   // never called
+
+constexpr int kRawSlices = 4;            // most slices of a 16-bit token that a thread keeps in registers (32 of them)
+
 // kSingle: K <= 4096 (one slice).  The thread's 16 features then stay in registers between the two passes, no
 // raw copy of x is kept in shared memory, and three CTAs fit on an SM (the call in progress and two
 // calls staging their weights behind it, or three independent calls).
@@ -631,7 +648,7 @@ gemv_decode_fast_kernel(GemvArgs a, FastGeom geo) {
   const int K = (int)a.K, Kp = geo.nslices * kSlice;                               // K rounded up to whole slices
   const uint32_t ring_alloc = geo.ring_bytes + (uint32_t)(a.K / 8) + 512u;         // lanes of a partial slice read past a row's end
   float* xf = reinterpret_cast<float*>(smem_raw + ring_alloc);                     // [Kp] raw x (not for kSingle)
-  int8_t* codes = reinterpret_cast<int8_t*>(smem_raw + ring_alloc + (kSingle ? 0 : (size_t)Kp * sizeof(float)));   // [Kp]
+  int8_t* codes = reinterpret_cast<int8_t*>(smem_raw + ring_alloc + (geo.x_in_smem ? (size_t)Kp * sizeof(float) : 0));   // [Kp]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t Kb = a.K / 8;
   const int rpw = geo.rpw, nslices = geo.nslices, depth = geo.depth;
@@ -726,9 +743,39 @@ gemv_decode_fast_kernel(GemvArgs a, FastGeom geo) {
 #pragma unroll
     for (int j = 0; j < 8; ++j) { v[j] = lo8[j]; v[8 + j] = hi8[j]; }
   };
+  // A 16-bit token of up to kRawSlices slices stays in registers as loaded (all loads issued at once,
+  // converted once for the sums and once more for the codes); longer or fp32 tokens go through shared
+  // memory as fp32, one slice at a time.
+  constexpr bool kRaw16 = !kSingle && sizeof(TX) == 2;
+  uint4 raw[kRaw16 ? kRawSlices : 1][2];
+  const bool in_regs = kRaw16 && !geo.x_in_smem;
+  auto from_raw = [&](int i, float (&v)[16]) {
+    float lo8[8], hi8[8];
+    unpack8<TX>(raw[kRaw16 ? i : 0][0], lo8);
+    unpack8<TX>(raw[kRaw16 ? i : 0][1], hi8);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { v[j] = lo8[j]; v[8 + j] = hi8[j]; }
+  };
   if (kSingle) {
     load16(0, xv);
     moments16(0, xv);
+  } else if (in_regs) {
+#pragma unroll
+    for (int i = 0; i < kRawSlices; ++i) {
+      if (i < nslices) {
+        const int k = i * kSlice + threadIdx.x * 8;
+        raw[kRaw16 ? i : 0][0] = __ldg(reinterpret_cast<const uint4*>(x + (kPartial ? min(k, K - 8) : k)));
+        raw[kRaw16 ? i : 0][1] = __ldg(reinterpret_cast<const uint4*>(x + (kPartial ? min(k + kSlice / 2, K - 8) : k + kSlice / 2)));
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < kRawSlices; ++i) {
+      if (i < nslices) {
+        float v[16];
+        from_raw(i, v);
+        moments16(i, v);
+      }
+    }
   } else {
 #pragma unroll 1
     for (int i = 0; i < nslices; ++i) {
@@ -813,6 +860,15 @@ gemv_decode_fast_kernel(GemvArgs a, FastGeom geo) {
   };
   if (kSingle) {
     quant16(0, xv);
+  } else if (in_regs) {
+#pragma unroll
+    for (int i = 0; i < kRawSlices; ++i) {
+      if (i < nslices) {
+        float v[16];
+        from_raw(i, v);
+        quant16(i, v);
+      }
+    }
   } else {
 #pragma unroll 1
     for (int i = 0; i < nslices; ++i) {
@@ -954,7 +1010,10 @@ cudaError_t run_fast(const GemvArgs& a, cudaStream_t s, int dev, int sms) {
   geo.nslices = (int)((a.K + kSlice - 1) / kSlice);
   const int64_t rows_per_cta = (a.N + sms - 1) / sms;
   const int64_t per_warp = (rows_per_cta + kGemvWarps - 1) / kGemvWarps;
-  const int64_t rmax = std::max<int64_t>(1, std::min<int64_t>(kBatchRows, 32768 / (kGemvWarps * Kb)));
+  int64_t rmax = std::max<int64_t>(1, std::min<int64_t>(kBatchRows, 32768 / (kGemvWarps * Kb)));
+  // long rows: when the CTA's whole slice fits the ring as one stage, take it as one (a warp then loads
+  // the codes of a K slice once for all of its rows instead of once per stage)
+  if (per_warp > rmax && per_warp <= kBatchRows && per_warp * kGemvWarps * Kb <= (int64_t)kRingBytes) rmax = per_warp;
   const int64_t nstages = (per_warp + rmax - 1) / rmax;
   if (nstages > 0x3FFFFFFF) return cudaErrorInvalidValue;
   geo.rows_per_cta = (int)rows_per_cta;
@@ -963,7 +1022,8 @@ cudaError_t run_fast(const GemvArgs& a, cudaStream_t s, int dev, int sms) {
   geo.stage_stride = (uint32_t)(geo.rpw * kGemvWarps * Kb);                      // a multiple of 4096, at most 32 KB
   const bool single = geo.nslices == 1;
   const size_t Kp = (size_t)geo.nslices * kSlice;
-  const size_t fixed = Kp * (single ? 1 : sizeof(float) + 1) + (size_t)Kb + 512;   // (raw x,) codes, slack beyond the ring
+  geo.x_in_smem = (!single && (sizeof(TX) != 2 || geo.nslices > kRawSlices)) ? 1 : 0;
+  const size_t fixed = Kp * (geo.x_in_smem ? sizeof(float) + 1 : 1) + (size_t)Kb + 512;   // (raw x,) codes, slack beyond the ring
   const size_t budget = std::min<size_t>(kRingBytes, 210 * 1024 - fixed);
   const int depth = std::max(1, std::min((int)(budget / geo.stage_stride), kMaxStages));
   geo.depth = (int)std::min<int64_t>(depth, nstages);
