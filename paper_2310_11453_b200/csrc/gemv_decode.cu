@@ -1159,7 +1159,7 @@ cudaError_t launch_gemv_decode(const GemvArgs& a, cudaStream_t s) {
 }  // namespace bl
 
 #ifdef BL_GEMV_STAMPS
-// Copies the stamp rings to the host: out must hold 2 * 64 records of (3 + 16) 64-bit words.
+// Copies the stamp rings to the host: out must hold 2 * 64 records of (3 + 32) 64-bit words.
 extern "C" int bitlinear_debug_gemv_stamps(unsigned long long* out, unsigned int* launches) {
   if (cudaDeviceSynchronize() != cudaSuccess) return 1;
   if (cudaMemcpyFromSymbol(out, bl::g_stamps, sizeof(bl::g_stamps)) != cudaSuccess) return 1;

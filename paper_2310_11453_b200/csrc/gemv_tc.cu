@@ -28,11 +28,13 @@
 //
 // Issue rate.  One thread issues a tcgen05.mma in about 63 clocks and a commit in about 67
 // whatever the shape, and several warps issue in parallel, so four issuer threads share the
-// work (two groups of chunks x two halves of the planes), each with accumulators of its own.
-// The expanders are two groups of four warps (one warp per lane quarter), each group filling
-// every other chunk of 256 weights into a ring of four A slots in tensor memory; the weights
-// are constants of the model, so the ring is filled and the CTA's weights are requested into L2
-// before the stream-order wait.
+// work (two planes each, every chunk), each plane's accumulator written by one thread only.
+// The expanders are two groups of four warps (one warp per lane quarter): group g forms planes
+// 4g..4g+3 of every chunk of 256 weights, two chunks per slot of its ring in tensor memory (three
+// slots with 16 tokens, two with 32, where the accumulators take twice the columns).  The weights
+// are constants of the model, so the rings are filled and the CTA's weights are requested into L2
+// before the stream-order wait.  tcgen05.st moves 128 bytes per clock and SM: the 454 KB of
+// expanded weights of a CTA (K 4096, 111 rows) are 3 550 clocks, the floor of this form.
 //
 // Waits: every mbarrier wait is bounded (tc_common.cuh); one that runs out raises the CTA's abort
 // flag, everybody falls through to the end, the status word of the workspace gets BL_ERR_TIMEOUT,
@@ -49,7 +51,7 @@ namespace {
 
 using namespace tc;
 
-constexpr int kTokMax = 32;              // tokens per pass (MMA N): 16, or 32 where their codes fit in shared memory
+                                         // tokens per pass (MMA N): 16, or 32 where their codes fit in shared memory
 constexpr int kQuantThreads = 256;        // with the product kernel's 384 threads on the same SM: registers for both
 constexpr int kQuantWarps = kQuantThreads / 32;
 constexpr int kMaxOctets = 6;            // 8-feature pieces per thread of the quantising kernel: K <= 12288

@@ -51,6 +51,15 @@ def test_packed_and_workspace_sizes():
     assert B.workspace_bytes(B.OP_FORWARD, 64, 3072, 768, 1) >= 64 * 768
     assert B.workspace_bytes(B.OP_FORWARD, 64, 3072, 768, 5) == 0      # K % (8 G) != 0
     assert B.workspace_bytes(B.OP_QUANT_ACT, 64, 1, 768, 65) == 0      # G too large
+    # small-batch decode with a workspace: a status block, then per pass of up to 32 tokens their codes
+    # (K bytes per token), gamma and the sum of the codes; enough for passes of 16 as well
+    for M, K in [(8, 4096), (16, 4096), (17, 4096), (32, 6144), (33, 8192), (40, 12288)]:
+        need = B.workspace_bytes(B.OP_GEMV_DECODE_BATCH, M, 16384, K, 1)
+        assert need % 256 == 0
+        assert need >= 256 + -(-M // 32) * 32 * (K + 8)
+        assert need >= 256 + -(-M // 16) * 16 * (K + 8)
+        assert need <= 512 + -(-M // 32) * 32 * (K + 8) + 256
+    assert B.workspace_bytes(B.OP_GEMV_DECODE_BATCH, 8, 16384, 4100, 1) == 0     # K % 8 != 0
 
 
 @pytest.mark.parametrize("layout,N,K", [(B.CANONICAL, 5, 40), (B.PREFILL, 130, 144), (B.PREFILL, 256, 256),
