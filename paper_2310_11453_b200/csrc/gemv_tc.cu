@@ -183,21 +183,6 @@ __global__ void __launch_bounds__(kQuantThreads, 2) decode_quant_kernel(QuantTok
   const float near = 0.5f - tau;
   const float lo_f = (a.mode == BL_ABSMAX) ? -(float)kCodeMax : 0.f;
 
-  if (threadIdx.x == 0) {
-    // gamma of Eq. 5 / 6 on x^ = (x - mean) rstd: only the final rescale reads it
-    float rstd = 1.f;
-    if (ln) {
-      const float var_f = fmaxf(fmaf(-off, off, t2 * a.inv_k), 0.f);
-      const float vv = var_f + a.ln_eps;
-      if (vv > 1e-30f && vv < 1e30f) {
-        const float y = rsqrtf(vv);
-        rstd = y * (1.5f - 0.5f * vv * y * y);
-      } else {
-        rstd = rstd_outside_fp32(vv);
-      }
-    }
-    reinterpret_cast<float*>(region + (size_t)a.nt * (size_t)a.K)[n] = span_f * rstd;
-  }
   // ---- Eq. 4 / 6: codes, written where the product kernel's MMAs read them ---------------------------
   int csum = 0;
 #pragma unroll
@@ -234,14 +219,27 @@ __global__ void __launch_bounds__(kQuantThreads, 2) decode_quant_kernel(QuantTok
       csum = __dp4a((int)w1, 0x01010101, csum);
     }
   }
-  csum = warp_sum(csum);
+  csum = __reduce_add_sync(0xFFFFFFFFu, csum);
   if (lane == 0) red_c[warp] = csum;
+  if (threadIdx.x == kQuantThreads - 32) {          // (a warp that does not close the kernel)
+    // gamma of Eq. 5 / 6 on x^ = (x - mean) rstd: only the final rescale reads it
+    float rstd = 1.f;
+    if (ln) {
+      const float var_f = fmaxf(fmaf(-off, off, t2 * a.inv_k), 0.f);
+      const float vv = var_f + a.ln_eps;
+      if (vv > 1e-30f && vv < 1e30f) {
+        const float y = rsqrtf(vv);
+        rstd = y * (1.5f - 0.5f * vv * y * y);
+      } else {
+        rstd = rstd_outside_fp32(vv);
+      }
+    }
+    reinterpret_cast<float*>(region + (size_t)a.nt * (size_t)a.K)[n] = span_f * rstd;
+  }
   __syncthreads();
-  if (threadIdx.x < kQuantWarps) {
-    int t = red_c[threadIdx.x];
-#pragma unroll
-    for (int o = kQuantWarps / 2; o > 0; o >>= 1) t += __shfl_xor_sync((1u << kQuantWarps) - 1u, t, o);
-    if (threadIdx.x == 0) reinterpret_cast<int*>(region + (size_t)a.nt * (size_t)a.K)[a.nt + n] = t;
+  if (warp == 0) {
+    const int t = __reduce_add_sync(0xFFFFFFFFu, lane < kQuantWarps ? red_c[lane] : 0);
+    if (lane == 0) reinterpret_cast<int*>(region + (size_t)a.nt * (size_t)a.K)[a.nt + n] = t;
   }
 }
 
