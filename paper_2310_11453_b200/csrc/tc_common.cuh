@@ -112,13 +112,30 @@ __device__ __forceinline__ uint32_t signs4(uint32_t word, int j) {
   return 0xFFFFFFFFu - 0xFEu * t;
 }
 
+// One 32-byte store (a whole sector) from a thread; dst must be 32-byte aligned.  A thread of the
+// epilogue owns a row of y, so a warp's store touches 32 rows: with 16-byte stores every access was half
+// a sector, and the stores of the bench GEMM cost a tenth of its time (93 us without them, 103 with).
+__device__ __forceinline__ void st_global_256(void* dst, const uint32_t (&w)[8]) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+}
+__device__ __forceinline__ bool aligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }
+
 template <typename TY>
 __device__ __forceinline__ void store_row32(TY* dst, const float (&v)[32], int64_t n0, int64_t N, bool vec_ok);
 
 template <>
 __device__ __forceinline__ void store_row32<float>(float* dst, const float (&v)[32], int64_t n0, int64_t N,
                                                    bool vec_ok) {
-  if (vec_ok) {
+  if (vec_ok && aligned32(dst)) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      uint32_t w[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) w[j] = __float_as_uint(v[8 * i + j]);
+      st_global_256(dst + 8 * i, w);
+    }
+  } else if (vec_ok) {
 #pragma unroll
     for (int i = 0; i < 8; ++i)
       *reinterpret_cast<float4*>(dst + 4 * i) = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
@@ -130,7 +147,18 @@ __device__ __forceinline__ void store_row32<float>(float* dst, const float (&v)[
 template <>
 __device__ __forceinline__ void store_row32<__half>(__half* dst, const float (&v)[32], int64_t n0, int64_t N,
                                                     bool vec_ok) {
-  if (vec_ok) {
+  if (vec_ok && aligned32(dst)) {
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      uint32_t w[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        __half2 h = __halves2half2(__float2half_rn(v[16 * i + 2 * j]), __float2half_rn(v[16 * i + 2 * j + 1]));
+        w[j] = *reinterpret_cast<uint32_t*>(&h);
+      }
+      st_global_256(dst + 16 * i, w);
+    }
+  } else if (vec_ok) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       uint32_t w[4];
@@ -149,7 +177,19 @@ __device__ __forceinline__ void store_row32<__half>(__half* dst, const float (&v
 template <>
 __device__ __forceinline__ void store_row32<__nv_bfloat16>(__nv_bfloat16* dst, const float (&v)[32], int64_t n0,
                                                            int64_t N, bool vec_ok) {
-  if (vec_ok) {
+  if (vec_ok && aligned32(dst)) {
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      uint32_t w[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        __nv_bfloat162 h = __halves2bfloat162(__float2bfloat16_rn(v[16 * i + 2 * j]),
+                                              __float2bfloat16_rn(v[16 * i + 2 * j + 1]));
+        w[j] = *reinterpret_cast<uint32_t*>(&h);
+      }
+      st_global_256(dst + 16 * i, w);
+    }
+  } else if (vec_ok) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       uint32_t w[4];
