@@ -112,11 +112,13 @@ __device__ __forceinline__ uint32_t signs4(uint32_t word, int j) {
   return 0xFFFFFFFFu - 0xFEu * t;
 }
 
-// One 32-byte store (a whole sector) from a thread; dst must be 32-byte aligned.  A thread of the
-// epilogue owns a row of y, so a warp's store touches 32 rows: with 16-byte stores every access was half
-// a sector, and the stores of the bench GEMM cost a tenth of its time (93 us without them, 103 with).
+// One 32-byte store (a whole sector) from a thread, not allocated in L1; dst must be 32-byte aligned.
+// A thread of the epilogue owns a row of y, so a warp's store touches 32 rows: with 16-byte stores every
+// access was half a sector, and the stores of the bench GEMM cost a tenth of its time (93 us without
+// them, 102 with; 96-97 with whole sectors, 94 when they also bypass L1, where they displaced what the
+// expander warps read).
 __device__ __forceinline__ void st_global_256(void* dst, const uint32_t (&w)[8]) {
-  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+  asm volatile("st.global.L1::no_allocate.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
                ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
 }
 __device__ __forceinline__ bool aligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }
