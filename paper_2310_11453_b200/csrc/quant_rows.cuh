@@ -190,7 +190,9 @@ __device__ __forceinline__ void row_store_codes_impl(const uint4* slot, int ni, 
     const int c = lane + 32 * i;
     Chunk<T> ch; float v[8];
     ch.load(slot, c); ch.unpack(v);
-    *reinterpret_cast<uint2*>(dst + (size_t)c * 8) = row_codes8<kClip>(v, map);
+    const uint2 cd = row_codes8<kClip>(v, map);
+    // (streamed out past L1: nothing on this SM reads the codes again; 1 % on the bench shape)
+    asm volatile("st.global.L1::no_allocate.v2.b32 [%0], {%1, %2};" ::"l"(dst + (size_t)c * 8), "r"(cd.x), "r"(cd.y) : "memory");
   }
 }
 template <typename T>
