@@ -41,8 +41,8 @@ INT8_TO_BF16 = 2.0                                   # nominal dense int8 : bf16
 # profiles/, taken with ncu on these same workloads.  A figure is valid only while its kernel is the
 # one that was profiled: set it to None when the kernel changes, until the capture is redone.
 NCU_TRAFFIC = {
-    "gemm_tc2_kernel": 54.2e6,                       # 36.5 MB read + 17.7 MB written (y largely still in L2)
-    "rows_tensor_fused": 70.3e6,                     # 67.2 MB read + 3.2 MB written (second pass from smem and L2)
+    "gemm_tc2_kernel": 70.6e6,                       # 37.1 MB read + 33.5 MB written (half of y still in L2)
+    "rows_tensor_fused": 70.9e6,                     # 67.2 MB read + 3.7 MB written (second pass from smem and L2)
     "gemv_decode_fast_kernel": 8.43e6,
     "reduce_partials + sign_pack_rows": 70.1e6,      # first pass 66.3 MB read, second pass served from L2
                                                      # (capture without cache flushes between the launches)
