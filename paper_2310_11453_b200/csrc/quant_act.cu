@@ -43,6 +43,7 @@ constexpr int kMaxStatCtas = 256;  // upper bound on the grid of the persistent 
 // Per-tensor workspace:
 //   status word (256 bytes reserved) | TensorScope | ScopePartial[kMaxStatCtas][BL_MAX_GROUPS] |
 //   arrival tags u64[kMaxStatCtas] | SegRecord[M*G].
+constexpr size_t kWsGenOff = 128;     // inside the status block: generation count of the fused kernel's meeting
 constexpr size_t kWsScopeOff = 256;
 constexpr size_t kWsPartialOff = kWsScopeOff + sizeof(TensorScope);
 constexpr size_t kWsTagOff = kWsPartialOff + (size_t)kMaxStatCtas * BL_MAX_GROUPS * sizeof(ScopePartial);
@@ -473,13 +474,15 @@ template <typename T>
 __global__ void __launch_bounds__(kRowWarps * 32, 1)
 rows_tensor_fused(const T* __restrict__ x, int64_t segments, int64_t K, int G, int Kg, int mode, float ln_eps,
                   double inv_kg, ScopePartial* __restrict__ partials, SegRecord* __restrict__ recs,
-                  unsigned long long* __restrict__ tags, unsigned long long tag, unsigned long long wait_tag,
+                  unsigned long long* __restrict__ tags, unsigned long long* __restrict__ generation,
+                  unsigned long long tag, unsigned long long wait_tag,
                   unsigned meet_polls, uint32_t* __restrict__ status, int clear_status, int8_t* __restrict__ x_q, float* __restrict__ gamma, float* __restrict__ eta) {
   extern __shared__ __align__(16) unsigned char stage[];
   __shared__ int counter1, counter2;
   __shared__ unsigned long long part_lo[BL_MAX_GROUPS], part_hi[BL_MAX_GROUPS];
   __shared__ double gam_s[BL_MAX_GROUPS], eta_s[BL_MAX_GROUPS];
   __shared__ unsigned long long copy_bar[kRowWarps][2];        // one mbarrier per warp and slot
+  __shared__ unsigned long long gen_s;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   if (threadIdx.x == 0) { counter1 = 0; counter2 = 0; }
   Staging sg = staging_init(stage, copy_bar, status);
@@ -487,6 +490,11 @@ rows_tensor_fused(const T* __restrict__ x, int64_t segments, int64_t K, int G, i
   __syncthreads();
   pdl_wait();
   pdl_launch_dependents();
+  // The tag is a launch parameter, so a captured graph replays it; the workspace's generation count,
+  // which CTA 0 advances after every meeting, makes what is published differ from launch to launch all
+  // the same.  Any starting value will do: all CTAs of a launch read the same one (it only changes after
+  // their meeting).  Visible to the whole CTA by the barriers ahead of the meeting.
+  if (threadIdx.x == 0) gen_s = *generation;
   if (clear_status && blockIdx.x == 0 && threadIdx.x == 0) *status = 0u;   // a timeout (seconds later) overwrites it
 
   const RowRange rg = cta_range(segments);
@@ -548,6 +556,9 @@ rows_tensor_fused(const T* __restrict__ x, int64_t segments, int64_t K, int G, i
   __syncthreads();
 
   // ---- the CTAs meet
+  const unsigned long long mix = gen_s * 0x9E3779B97F4A7C15ull;
+  tag ^= mix;
+  wait_tag ^= mix;
   if (threadIdx.x == 0) { __threadfence(); st_release_u64(tags + blockIdx.x, tag); }
   bool here = true;
   if (threadIdx.x < gridDim.x) {
@@ -568,6 +579,7 @@ rows_tensor_fused(const T* __restrict__ x, int64_t segments, int64_t K, int G, i
     if (threadIdx.x == 0) atomicExch(status, (uint32_t)BL_ERR_TIMEOUT);
     return;
   }
+  if (blockIdx.x == 0 && threadIdx.x == 0) *generation = gen_s + 1;   // every CTA has read it: all have arrived
 
   // ---- gamma / eta of every group from all CTAs' extremes
   for (int g = warp; g < G; g += kRowWarps) {
@@ -656,6 +668,7 @@ cudaError_t launch_fused(const QuantArgs& a, cudaStream_t s, const T* x, int64_t
   }
   if ((int64_t)grid > (int64_t)cap) grid = (unsigned)cap;
   unsigned long long* tags = reinterpret_cast<unsigned long long*>(reinterpret_cast<char*>(a.ws) + kWsTagOff);
+  unsigned long long* generation = reinterpret_cast<unsigned long long*>(reinterpret_cast<char*>(a.ws) + kWsGenOff);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
   cfg.blockDim = dim3(kRowWarps * 32);
@@ -677,13 +690,13 @@ cudaError_t launch_fused(const QuantArgs& a, cudaStream_t s, const T* x, int64_t
   const unsigned long long wait_tag = g_debug_meet_skew.load(std::memory_order_relaxed) ? ~tag : tag;
   const int clear = a.keep_status ? 0 : 1;
   e = cudaLaunchKernelEx(&cfg, kern, x, segments, a.K, a.G, Kg, (int)a.mode, a.ln_eps, inv_kg, partials, recs, tags,
-                         tag, wait_tag, meet_polls, status, clear, a.x_q, a.gamma, a.eta);
+                         generation, tag, wait_tag, meet_polls, status, clear, a.x_q, a.gamma, a.eta);
   if (e != cudaSuccess && cfg.numAttrs == 2) {
     (void)cudaGetLastError();
     with_pdl.store(0);
     cfg.numAttrs = 1;
     e = cudaLaunchKernelEx(&cfg, kern, x, segments, a.K, a.G, Kg, (int)a.mode, a.ln_eps, inv_kg, partials, recs, tags,
-                           tag, wait_tag, meet_polls, status, clear, a.x_q, a.gamma, a.eta);
+                           generation, tag, wait_tag, meet_polls, status, clear, a.x_q, a.gamma, a.eta);
   }
   return e;
 }

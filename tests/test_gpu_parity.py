@@ -219,6 +219,33 @@ def test_quant_act(M, K, G, dtype, mode, gran, outliers, relu):
             assert torch.equal(out[key], with_ws[key]) and torch.equal(out[key], no_ws[key])
 
 
+def test_quant_act_per_tensor_replayed_from_a_graph_on_new_data():
+    # The fused per-tensor kernel's CTAs meet over tags in the workspace.  A captured graph replays the
+    # same launch parameters, so what a CTA publishes must still differ from one replay to the next (a
+    # generation count in the workspace): otherwise the second replay would take the first one's tags
+    # for arrivals and compute gamma from stale or half-written partial extremes.
+    M, K = 600, 4096
+    xa = synth.make_x(M, K, torch.bfloat16, seed=5, outliers=True)
+    xb = (synth.make_x(M, K, torch.bfloat16, seed=6, outliers=False).float() * 3.0 + 0.5).to(torch.bfloat16)
+    x = xa.to(DEV).clone()
+    out = dict(x_q=torch.empty((M, K), dtype=torch.int8, device=DEV), gamma=torch.empty(1, device=DEV),
+               eta=torch.empty(1, device=DEV))
+    ws = torch.empty(B.workspace_bytes(B.OP_QUANT_ACT, M, 1, K, 1), dtype=torch.uint8, device=DEV)
+    B.quant_act(x, gran=B.PER_TENSOR, out=out, ws=ws)                # warm-up outside the capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        B.quant_act(x, gran=B.PER_TENSOR, out=out, ws=ws)
+    for host in (xa, xb, xa, xb):
+        x.copy_(host.to(DEV))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert B.ws_status(ws) == B.OK
+        ref = O.quant_act(as_f32_np(host), G=1, mode=O.ABSMAX, gran=O.PER_TENSOR, ln_eps=1e-5)
+        check_codes(out["x_q"].cpu().numpy(), ref["codes"], x=as_f32_np(host), G=1)
+        check_scalars(out["gamma"].cpu().numpy(), ref["gamma"])
+
+
 def test_quant_act_per_tensor_status_word_and_workspace_reuse():
     # The per-tensor path keeps its status word in the workspace; reusing one (uninitialised)
     # workspace for calls of different shapes must leave it clear and the results unchanged.
