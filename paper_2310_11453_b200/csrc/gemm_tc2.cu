@@ -344,7 +344,14 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap map_x, GemmArgs a, int tx_by
           if (kMode == 0) {
             if (m_ok) {
               int32_t* dst = a.acc + ((int64_t)g * a.M + m) * a.N + n0;
-              if (n0 + 32 <= a.N && (a.N & 3) == 0) {
+              if (n0 + 32 <= a.N && (a.N & 3) == 0 && aligned32(dst)) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  const uint32_t w[8] = {r[8 * i], r[8 * i + 1], r[8 * i + 2], r[8 * i + 3],
+                                         r[8 * i + 4], r[8 * i + 5], r[8 * i + 6], r[8 * i + 7]};
+                  st_global_256(dst + 8 * i, w);
+                }
+              } else if (n0 + 32 <= a.N && (a.N & 3) == 0) {
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
                   *reinterpret_cast<uint4*>(dst + 4 * i) = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
