@@ -399,10 +399,7 @@ bl_status bitlinear_gemv_decode_batch_ws(const void* x, bl_dtype xt, int64_t M, 
   if (eta_correction && mode != BL_ETA) return BL_ERR_UNSUPPORTED;
   if (!aligned16(x) || !aligned16(W_packed) || !aligned16(y)) return BL_ERR_ALIGN;
   GemvArgs a{x, xt, K, N, G, mode, ln_eps, eta_correction ? 1 : 0, W_packed, beta, rowsum, y, yt};
-  // Below 8 tokens the one-kernel form is as fast or faster where it takes the shape (measured on
-  // K 4096, N 16384: 9.1 / 9.9 us for 2 / 4 tokens against 10.4 / 10.6; 11.7 against 10.8 at 8).
-  const bool one_kernel = M < 8 && gemv_batch_supported(M, K, N, G);
-  if (!one_kernel && gemv_tc_supported(M, K, N, G, eta_correction)) {
+  if (gemv_tc_supported(M, K, N, G, eta_correction)) {
     if (!ws || ws_bytes < bitlinear_workspace_bytes(BL_OP_GEMV_DECODE_BATCH, M, N, K, G)) return BL_ERR_WORKSPACE;
     if (!aligned16(ws)) return BL_ERR_ALIGN;
     return launch_gemv_tc(a, M, ws, (cudaStream_t)stream) == cudaSuccess ? BL_OK : BL_ERR_CUDA;

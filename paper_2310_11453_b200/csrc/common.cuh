@@ -195,6 +195,8 @@ cudaError_t gemv_decode_take_fallbacks(unsigned int* out);   // warps that read 
 // The same for M tokens (x [M,K], y [M,N]) sharing one pass over the weights per 8 tokens.
 cudaError_t launch_gemv_batch(const GemvArgs& a, int64_t M, cudaStream_t s);
 bool gemv_batch_supported(int64_t M, int64_t K, int64_t N, int G);
+cudaError_t launch_gemv_batch_pre(const GemvArgs& g, int64_t M, const int8_t* codes, const float* gamma, const int* csum,
+                                  cudaStream_t s);   // the same kernel on tokens quantised earlier on the stream
 // The same with a workspace: tokens quantised once by a kernel of their own, the product on the
 // tcgen05 tensor cores, 16 tokens per pass over the weights (gemv_tc.cu).
 cudaError_t launch_gemv_tc(const GemvArgs& a, int64_t M, void* ws, cudaStream_t s);

@@ -73,6 +73,9 @@ struct BatchArgs {
   int stage_tokens;                      // the raw tokens fit in shared memory beside the codes
   double inv_kg;                         // 1 / K_g (a double-precision division per thread otherwise)
   uint32_t* clear_status;                // when set: a status word this launch clears, in stream order
+  const int8_t* pre_codes;               // when set (one group): the tokens' codes [M][K], their gamma [M] and code
+  const float* pre_gamma;                // sums [M], the work of a kernel earlier on the stream; the tokens are
+  const int* pre_csum;                   // then not quantised here
 };
 
 // The four A words of K block b for this lane: rows g and g + 8, words qd and 4 + qd of the block.
@@ -135,7 +138,20 @@ gemv_batch_kernel(BatchArgs a) {
   pdl_wait();
   if (a.clear_status != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *a.clear_status = 0u;
 
-  // ---- 2. LN + Quant of the tokens
+  // ---- 2. LN + Quant of the tokens (or their codes as another kernel left them)
+  if (a.pre_codes != nullptr) {
+    const int pieces_per_row = (int)(a.K / 16);
+    for (int i = threadIdx.x; i < a.M * pieces_per_row; i += kBatchWarps * 32) {
+      const int tok = i / pieces_per_row, p = i - tok * pieces_per_row;
+      cp_async16(codes + (int64_t)tok * stride + (int64_t)p * 16, a.pre_codes + (int64_t)tok * a.K + (int64_t)p * 16);
+    }
+    if (threadIdx.x < a.M) {
+      sh.gamma[threadIdx.x][0] = a.pre_gamma[threadIdx.x];
+      sh.eta[threadIdx.x][0] = 0.f;
+      sh.csum[threadIdx.x][0] = a.pre_csum[threadIdx.x];
+    }
+    asm volatile("cp.async.wait_all;" ::: "memory");
+  } else {
   if (a.stage_tokens) {
     const uint4* src = reinterpret_cast<const uint4*>(a.x);
     uint4* dst = reinterpret_cast<uint4*>(raw);
@@ -260,6 +276,7 @@ gemv_batch_kernel(BatchArgs a) {
       }
     }
   }
+  }
   __syncthreads();
 
   // ---- 3. rows.  Lanes of absent tokens read zeros.
@@ -359,8 +376,12 @@ cudaError_t run2(BatchArgs a, cudaStream_t s) {
   if (e != cudaSuccess) return e;
   if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
   const int64_t tiles = a.N / kTileRows;
-  const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
-  a.stage_tokens = batch_smem(a.M, a.K, sizeof(TX), true) <= kSmemBudget ? 1 : 0;
+  // With the tokens quantised by a kernel of one CTA per token just ahead of this one, leave that kernel its
+  // SMs: a CTA here takes every register of an SM, so one that had to share would only start when the
+  // other kernel's CTA has gone, without the head start on its weights.
+  const int64_t usable = a.pre_codes != nullptr && sms > 2 * a.M ? sms - a.M : sms;
+  const unsigned grid = (unsigned)(tiles < usable ? tiles : usable);
+  a.stage_tokens = (a.pre_codes == nullptr && batch_smem(a.M, a.K, sizeof(TX), true) <= kSmemBudget) ? 1 : 0;
   const size_t smem = batch_smem(a.M, a.K, sizeof(TX), a.stage_tokens != 0);
   if ((e = cudaFuncSetAttribute(gemv_batch_kernel<TX, TY>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) !=
       cudaSuccess)
@@ -401,6 +422,7 @@ cudaError_t launch_gemv_batch(const GemvArgs& g, int64_t M, cudaStream_t s) {
     a.stage_tokens = 0;
     a.inv_kg = 1.0 / (double)(g.K / g.G);
     a.clear_status = m0 == 0 ? g.clear_status : nullptr;
+    a.pre_codes = nullptr; a.pre_gamma = nullptr; a.pre_csum = nullptr;
     cudaError_t e = cudaErrorInvalidValue;
     switch (g.xt) {
       case BL_F32: e = run1<float>(a, g.yt, s); break;
@@ -410,6 +432,27 @@ cudaError_t launch_gemv_batch(const GemvArgs& g, int64_t M, cudaStream_t s) {
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;
+}
+
+// One launch for up to 8 tokens (one group) whose codes [M][K], gamma [M] and code sums [M] an earlier
+// kernel on the stream has written.
+cudaError_t launch_gemv_batch_pre(const GemvArgs& g, int64_t M, const int8_t* codes, const float* gamma, const int* csum,
+                                  cudaStream_t s) {
+  if (M < 1 || M > kBatchTokens || g.G != 1) return cudaErrorInvalidValue;
+  BatchArgs a;
+  a.x = g.x; a.M = (int)M;
+  a.K = g.K; a.N = g.N; a.G = 1; a.mode = (int)g.mode; a.ln_eps = g.ln_eps; a.eta_correction = 0;
+  a.W_packed = g.W_packed; a.beta = g.beta; a.rowsum = g.rowsum; a.y = g.y;
+  a.stage_tokens = 0;
+  a.inv_kg = 1.0 / (double)g.K;
+  a.clear_status = nullptr;
+  a.pre_codes = codes; a.pre_gamma = gamma; a.pre_csum = csum;
+  switch (g.xt) {
+    case BL_F32: return run1<float>(a, g.yt, s);
+    case BL_F16: return run1<__half>(a, g.yt, s);
+    case BL_BF16: return run1<__nv_bfloat16>(a, g.yt, s);
+  }
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace bl

@@ -83,6 +83,7 @@ struct QuantTokArgs {
   const void* x; int64_t K; int mode; float ln_eps;
   float inv_k; double inv_k_d;
   int nt;                   // tokens per pass
+  int row_major;            // codes as plain rows [token][K] (for the bit-plane kernel) instead of MMA tiles
   uint8_t* passes;          // workspace behind the status block
   uint32_t* status;         // cleared here (in stream order); the product kernels only ever raise it
 };
@@ -212,9 +213,13 @@ __global__ void __launch_bounds__(kQuantThreads, 2) decode_quant_kernel(QuantTok
       }
       const uint32_t w0 = __byte_perm(__byte_perm(tb[0], tb[1], 0x0040), __byte_perm(tb[2], tb[3], 0x0040), 0x5410);
       const uint32_t w1 = __byte_perm(__byte_perm(tb[4], tb[5], 0x0040), __byte_perm(tb[6], tb[7], 0x0040), 0x5410);
-      const uint32_t offb = code_offset4(8 * c, n, (int)(a.K / 128));       // features 8c..8c+3; 8c+4..8c+7 are the next plane, 32 bytes on
-      *reinterpret_cast<uint32_t*>(region + offb) = w0;
-      *reinterpret_cast<uint32_t*>(region + (offb ^ 32u)) = w1;
+      if (a.row_major) {
+        *reinterpret_cast<uint2*>(region + (size_t)n * (size_t)a.K + (size_t)c * 8) = make_uint2(w0, w1);
+      } else {
+        const uint32_t offb = code_offset4(8 * c, n, (int)(a.K / 128));     // features 8c..8c+3; 8c+4..8c+7 are the next plane, 32 bytes on
+        *reinterpret_cast<uint32_t*>(region + offb) = w0;
+        *reinterpret_cast<uint32_t*>(region + (offb ^ 32u)) = w1;
+      }
       csum = __dp4a((int)w0, 0x01010101, csum);
       csum = __dp4a((int)w1, 0x01010101, csum);
     }
@@ -529,7 +534,7 @@ cudaError_t run(const GemvArgs& a, int64_t M, void* ws, cudaStream_t s) {
     if (dev < 64) configured[dev].store(1, std::memory_order_release);
   }
   uint8_t* base = reinterpret_cast<uint8_t*>(ws);
-  QuantTokArgs qa{a.x, a.K, (int)a.mode, a.ln_eps, (float)(1.0 / (double)a.K), 1.0 / (double)a.K, nt, base + kStatusBytes,
+  QuantTokArgs qa{a.x, a.K, (int)a.mode, a.ln_eps, (float)(1.0 / (double)a.K), 1.0 / (double)a.K, nt, 0, base + kStatusBytes,
                   reinterpret_cast<uint32_t*>(base)};
   const int64_t per_thread = (a.K / 8 + kQuantThreads - 1) / kQuantThreads;
   if (per_thread <= 2) e = launch_pdl(decode_quant_kernel<TX, 2>, dim3((unsigned)M), dim3(kQuantThreads), 0, s, qa);
@@ -548,8 +553,28 @@ cudaError_t run(const GemvArgs& a, int64_t M, void* ws, cudaStream_t s) {
   return cudaSuccess;
 }
 
+// Up to 8 tokens: the same quantising kernel (codes as plain rows), then the bit-plane kernel of
+// gemv_batch.cu told to take codes, gamma and the code sums from the workspace instead of computing them
+// in every CTA.
+template <typename TX>
+cudaError_t run_small(const GemvArgs& a, int64_t M, void* ws, cudaStream_t s) {
+  uint8_t* base = reinterpret_cast<uint8_t*>(ws);
+  uint8_t* region = base + kStatusBytes;
+  QuantTokArgs qa{a.x, a.K, (int)a.mode, a.ln_eps, (float)(1.0 / (double)a.K), 1.0 / (double)a.K, (int)M, 1, region,
+                  reinterpret_cast<uint32_t*>(base)};
+  const int64_t per_thread = (a.K / 8 + kQuantThreads - 1) / kQuantThreads;
+  cudaError_t e;
+  if (per_thread <= 2) e = launch_pdl(decode_quant_kernel<TX, 2>, dim3((unsigned)M), dim3(kQuantThreads), 0, s, qa);
+  else if (per_thread <= 4) e = launch_pdl(decode_quant_kernel<TX, 4>, dim3((unsigned)M), dim3(kQuantThreads), 0, s, qa);
+  else e = launch_pdl(decode_quant_kernel<TX, 6>, dim3((unsigned)M), dim3(kQuantThreads), 0, s, qa);
+  if (e != cudaSuccess) return e;
+  const float* gamma = reinterpret_cast<const float*>(region + (size_t)M * (size_t)a.K);
+  return launch_gemv_batch_pre(a, M, reinterpret_cast<const int8_t*>(region), gamma, reinterpret_cast<const int*>(gamma) + M, s);
+}
+
 template <typename TX>
 cudaError_t run1(const GemvArgs& a, int64_t M, void* ws, cudaStream_t s) {
+  if (M <= 8) return run_small<TX>(a, M, ws, s);
   switch (a.yt) {
     case BL_F32: return run<TX, float>(a, M, ws, s);
     case BL_F16: return run<TX, __half>(a, M, ws, s);
@@ -562,7 +587,7 @@ cudaError_t run1(const GemvArgs& a, int64_t M, void* ws, cudaStream_t s) {
 
 bool gemv_tc_supported(int64_t M, int64_t K, int64_t N, int G, int eta_correction) {
   return M >= 2 && G == 1 && !eta_correction && K % 256 == 0 && N % 16 == 0 && N > 0 &&
-         K <= (int64_t)kMaxOctets * kQuantThreads * 8;
+         K <= (int64_t)kMaxOctets * kQuantThreads * 8 && (M > 8 || gemv_batch_supported(M, K, N, G));
 }
 
 size_t gemv_tc_ws_bytes(int64_t M, int64_t K) {

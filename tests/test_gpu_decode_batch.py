@@ -31,28 +31,31 @@ def test_gemv_decode_batch(M, K, N, G, dtype, mode, relu):
 # The same call with a workspace: tokens quantised by a kernel of their own, the product on the
 # tcgen05 tensor cores for G == 1 without the eta correction (other cases: the kernel above).
 @pytest.mark.parametrize("M,K,N,G,dtype,mode,relu", [
-    (8, 4096, 16384, 1, "f16", "absmax", False),     # config c2's layer, 8 tokens: 148 CTAs of 111 rows
+    (8, 4096, 16384, 1, "f16", "absmax", False),     # config c2's layer, 8 tokens: quantising kernel + bit-plane kernel
+    (9, 4096, 16384, 1, "f16", "absmax", False),     # 9 tokens: quantising kernel + tensor-core kernel, 148 CTAs of 111 rows
     (16, 4096, 16384, 1, "bf16", "absmax", False),   # a full pass of 16 tokens
-    (8, 256, 16, 1, "f32", "absmax", False),         # smallest shape: one chunk (half a slot), CTAs of one row
+    (2, 256, 16, 1, "f32", "absmax", False),         # smallest shape
+    (12, 256, 16, 1, "f32", "absmax", False),        # the same on the tensor cores: one chunk (half a slot), CTAs of one row
     (9, 1024, 48, 1, "bf16", "eta", True),           # eta form without the correction; the second half of the codes is used
     (37, 2048, 160, 1, "f16", "absmax", False),      # passes of 32 tokens: a full one and a ragged one of 5
     (32, 4096, 16384, 1, "f16", "absmax", False),    # one pass of 32 tokens at config c2's layer
     (17, 6144, 256, 1, "bf16", "eta", True),         # the largest K with 32 tokens per pass; 17 tokens: three of four token blocks
     (20, 8192, 64, 1, "f16", "absmax", False),       # more than 16 tokens with K too large for 32 per pass: two passes of 16
     (11, 8192, 20480, 1, "bf16", "absmax", False),   # 160 CTAs of 128 rows: more CTAs than SMs
-    (8, 12288, 64, 1, "f32", "absmax", False),       # the largest K: six pieces per thread of the quantiser
+    (10, 12288, 64, 1, "f32", "absmax", False),      # the largest K: six pieces per thread of the quantiser
+    (5, 12288, 64, 1, "f32", "eta", True),           # the same with the bit-plane kernel
     (10, 768, 3072, 1, "f32", "absmax", False),      # 125M-shaped: an odd number of chunks
-    (4, 4096, 1024, 1, "f16", "absmax", False),      # fewer than 8 tokens: the kernel without a workspace
-    (9, 1024, 48, 2, "bf16", "eta", True),           # groups: likewise
-    (8, 16384, 48, 1, "f16", "absmax", False),       # K too large for the tensor-core form: likewise
+    (4, 4096, 1024, 1, "f16", "absmax", False),      # few tokens, few tiles
+    (9, 1024, 48, 2, "bf16", "eta", True),           # groups: the kernel without a workspace
+    (8, 16384, 48, 1, "f16", "absmax", False),       # K too large for the quantising kernel: likewise
 ])
 def test_gemv_decode_batch_ws(M, K, N, G, dtype, mode, relu):
     ws = torch.empty(B.workspace_bytes(B.OP_GEMV_DECODE_BATCH, M, N, K, G) + 256, dtype=torch.uint8, device=DEV)
 
     def call(*args, **kw):
         return B.gemv_decode_batch_ws(*args, ws=ws, **kw)
-    # below 8 tokens the call runs another kernel: same bits are promised among batches of 8 or more
-    run_batch_case(call, M, K, N, G, dtype, mode, relu, same_bits_from=8 if (G == 1 and K <= 12288) else 2)
+    # every token is quantised by the same kernel whichever product kernel follows: same bits for any batch
+    run_batch_case(call, M, K, N, G, dtype, mode, relu)
     assert B.ws_status(ws) == B.OK
 
 
