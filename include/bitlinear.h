@@ -292,18 +292,20 @@ bl_status bitlinear_gemv_decode_batch(const void* x, bl_dtype xt, int64_t M, int
                                       const uint8_t* W_packed, const float* beta, const int32_t* rowsum,
                                       void* y, bl_dtype yt, void* stream);
 
-/* bitlinear_gemv_decode_batch with a workspace (Sec. 2.1, Eq. 12, 4-7, 11 per token), for G == 1 and
- * eta_correction == 0, M >= 8 and K <= 12288: two kernels per call.  The first quantises the tokens
- * once (one CTA per token; LN statistics, gamma / eta, codes: the fp32 arithmetic of the kernel
- * of bitlinear_gemv_decode) into the workspace; the second streams the packed weights once per 32
- * tokens (per 16 when K > 6144) and multiplies on the tcgen05 tensor cores (weight bit planes
- * written to tensor memory as the A operand, int32 accumulators, exact), so the time of a call
- * depends little on M up to 32.
- * A token's result does not depend on what else is in the batch as long as the batch stays on the
- * same side of 8 tokens (same bits).  Fewer than 8 tokens, other shapes, G > 1 and eta_correction
- * are handed to the kernel of bitlinear_gemv_decode_batch where it takes the shape (of the
- * workspace only the status word is used: cleared; its shape rules apply; for fewer than 8 tokens
- * it is as fast or faster); M == 1 to that of bitlinear_gemv_decode.
+/* bitlinear_gemv_decode_batch with a workspace (Sec. 2.1, Eq. 12, 4-7, 11 per token), for G == 1,
+ * eta_correction == 0, M >= 2 and K <= 12288: two kernels per call.  The first quantises the tokens
+ * once (one CTA per token; LN statistics, gamma / eta, codes: the fp32 arithmetic of the kernel of
+ * bitlinear_gemv_decode) into the workspace.  The second streams the packed weights once and
+ * multiplies: for up to 8 tokens the bit-plane kernel of bitlinear_gemv_decode_batch, told to take
+ * codes, gamma and code sums from the workspace instead of quantising every token in every CTA; for
+ * more, the tcgen05 tensor cores (weight bit planes written to tensor memory as the A operand, int32
+ * accumulators, exact), one pass per 32 tokens (per 16 when K > 6144), so that the time of a call
+ * depends little on M up to 32.  A token's result does not depend on what else is in the batch, nor
+ * on which of the two product kernels ran (same bits).  Other shapes, G > 1 and eta_correction are
+ * handed to bitlinear_gemv_decode_batch's own path where it takes the shape (of the workspace only
+ * the status word is used: cleared; its shape rules apply); M == 1 to the kernel of
+ * bitlinear_gemv_decode, whose sums run in another order (same codes up to the tolerated ties,
+ * gamma to the last bit or so).
  *   x [M,K] of dtype xt;  y [M,N] of dtype yt;  W_packed in DECODE layout, read ahead of stream
  *   order as there.  K % 256 == 0, N % 16 == 0.
  * Workspace: BL_OP_GEMV_DECODE_BATCH (device memory, 16-byte aligned; its first word is the status
