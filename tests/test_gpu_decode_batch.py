@@ -134,6 +134,29 @@ def test_gemv_decode_batch_integer_definition_exactly():
     assert np.allclose(y.cpu().numpy(), want, rtol=3e-7, atol=0)
 
 
+@pytest.mark.parametrize("M", [6, 12, 32])
+def test_gemv_decode_batch_ws_integer_definition_exactly(M):
+    # As above through the workspace form: 6 tokens take the bit-plane kernel, 12 and 32 the tensor cores
+    # (one pass of 16, one of 32).  With LN skipped and gamma planted at 128 the codes are the inputs, so y
+    # must be the oracle's integer matmul times beta, to the last bit of the one float multiplication.
+    K, N = 1024, 96
+    codes = synth.make_codes(M, K, seed=9 + M)
+    x = codes.to(torch.float32)
+    x[:, 0] = 128.0                                                  # gamma = 128, its code clips to 127
+    W = synth.make_w(N, K, torch.float32, seed=9)
+    w_ref = O.binarize(W.numpy())
+    w_gpu = B.binarize_pack(W.to(DEV), layout=B.DECODE)
+    torch.cuda.synchronize()
+    ws = torch.empty(B.workspace_bytes(B.OP_GEMV_DECODE_BATCH, M, N, K, 1), dtype=torch.uint8, device=DEV)
+    y = B.gemv_decode_batch_ws(x.to(DEV), w_gpu["W_packed"], w_gpu["beta"], N, ln_eps=-1.0, out_dtype=torch.float32, ws=ws)
+    assert B.ws_status(ws) == B.OK
+    c = codes.numpy().copy()
+    c[:, 0] = 127
+    acc = O.matmul(c, w_ref["bits"])[0].astype(np.float64)
+    want = (acc * float(w_gpu["beta"][0])).astype(np.float32)
+    assert np.allclose(y.cpu().numpy(), want, rtol=3e-7, atol=0)
+
+
 def test_gemv_decode_batch_argument_checks():
     x = torch.zeros((2, 384), dtype=torch.float16, device=DEV)
     w = torch.zeros(64, dtype=torch.uint8, device=DEV)
