@@ -120,8 +120,12 @@ __global__ void __launch_bounds__(kQuantThreads, 2) decode_quant_kernel(QuantTok
   const int64_t m = blockIdx.x;
   const int n = (int)(m % a.nt);
   uint8_t* region = a.passes + (size_t)(m / a.nt) * pass_bytes(a.K, a.nt);
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");     // the product kernel may start on the weights
+  // The product kernel may start on the weights.  Measured: the bit-plane kernel does best released at
+  // once, the tensor-core kernel released once this kernel's own stream-order wait has returned (its 148
+  // CTAs then do not set up and prefetch while the kernel before this one is still finishing).
+  if (a.row_major) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (!a.row_major) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (m == 0 && threadIdx.x == 0) *a.status = 0u;
   const uint4* slot = reinterpret_cast<const uint4*>(reinterpret_cast<const TX*>(a.x) + m * a.K);
   const int octets = (int)(a.K / 8);
